@@ -1,0 +1,252 @@
+/*
+ * tasc.h -- C ABI of the B200 (sm_100a) implementation of one batched n-gram
+ * speculative-decoding step (TASC-draft; paper Sections 5.1 and 5.2).
+ *
+ * Conventions
+ *   - Plain C.  Every call returns a tasc_status (0 = OK, negative = error);
+ *     nothing throws, aborts or traps across this boundary.
+ *   - "device" pointers are CUDA global-memory addresses of the current device;
+ *     "host" pointers are ordinary process memory.  Each argument says which.
+ *   - tasc_stream is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Step calls (tasc_draft, tasc_verify_step, tasc_prefill) only enqueue work
+ *     on that stream and return; they allocate nothing.  Device-side problems
+ *     (a KV position outside the block table, a wait that ran out) are recorded
+ *     in a status word inside the caller's workspace and read by
+ *     tasc_poll_status, which synchronises the stream.
+ *   - The caller owns weights, KV pool, block table, token buffers and the
+ *     workspace.  The library owns only what tasc_drafter_build and
+ *     tasc_model_create allocate, released by the matching destroy call.
+ *   - Token ids are int32, document offsets int64.
+ */
+#ifndef TASC_H
+#define TASC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t tasc_status;
+#define TASC_OK          0
+#define TASC_EINVAL    (-1)   /* bad argument (null pointer, size out of range, unsupported shape) */
+#define TASC_ENOMEM    (-2)   /* device or host allocation failed */
+#define TASC_ECUDA     (-3)   /* a CUDA runtime / driver call failed */
+#define TASC_ECAPACITY (-4)   /* a hash table or output buffer is too small */
+#define TASC_ENOKV     (-5)   /* a KV position falls outside the sequence's block table */
+#define TASC_ETIMEOUT  (-6)   /* a bounded device-side wait ran out */
+
+#define TASC_MAX_ORDER   5    /* largest context length n_max of the n-gram models */
+#define TASC_MAX_ROWS   16    /* largest k + 1 (rows verified per sequence per step) */
+#define TASC_VOCAB_BITS 20    /* token ids must be < 2^20 (six ids + order are packed in 128 bits) */
+
+#define TASC_F32   0
+#define TASC_BF16  1
+
+typedef void* tasc_stream;
+typedef struct tasc_drafter tasc_drafter;
+typedef struct tasc_model tasc_model;
+
+/* One surviving element of a pruned n-gram model M_n: context of n tokens -> next token, count. */
+typedef struct {
+    int32_t  n;                      /* context length, 1..n_max */
+    int32_t  ctx[TASC_MAX_ORDER];    /* ctx[0..n-1], oldest first; unused slots are -1 */
+    int32_t  next;
+    uint32_t count;
+} tasc_ngram_entry;
+
+/* ------------------------------------------------------------------ drafter */
+
+/*
+ * Build the corpus n-gram drafter p_corp (Section 5.2: n-gram models M_n, n <= n_max,
+ * from the n-gram frequencies of the task's output corpus, each pruned of elements
+ * whose frequency is below p_min; plus the most frequent token as the last resort).
+ * n is the context length; n-grams do not cross document boundaries.
+ *
+ *   corpus_tokens  device, int32[doc_offsets[n_docs]], every id in [0, vocab)
+ *   doc_offsets    device, int64[n_docs + 1], non-decreasing, doc_offsets[0] = 0
+ *   n_max          1..TASC_MAX_ORDER;  p_min >= 1 (absolute count threshold)
+ *   vocab          <= 2^TASC_VOCAB_BITS
+ *   out            host; receives a handle owning device tables (tasc_drafter_destroy)
+ * Synchronises the stream before returning.  Errors: EINVAL, ENOMEM, ECUDA,
+ * ECAPACITY (internal table overflow; not expected for valid input).
+ */
+tasc_status tasc_drafter_build(const int32_t* corpus_tokens, const int64_t* doc_offsets, int64_t n_docs,
+                               int32_t n_max, int32_t p_min, int32_t vocab, tasc_stream stream,
+                               tasc_drafter** out);
+
+/*
+ * Canonical dump of the pruned models: entries sorted by (n, ctx, next).
+ *   out        host, room for cap entries (may be NULL when cap = 0 to query the size)
+ *   n_entries  host, receives the total number of entries (even if cap is smaller -> ECAPACITY)
+ *   fallback_token  host, receives the most frequent corpus token (smallest id on ties)
+ */
+tasc_status tasc_drafter_export(const tasc_drafter* d, tasc_ngram_entry* out, int64_t cap, int64_t* n_entries,
+                                int32_t* fallback_token);
+
+tasc_status tasc_drafter_destroy(tasc_drafter* d);
+
+/*
+ * Draft k tokens per sequence from p_mixed = lambda p_corp + (1 - lambda) p_prompt
+ * (Section 5.2, mixture equation), lambda = lambda_num / lambda_den, argmax with the
+ * smallest token id on ties, evaluated exactly in 64-bit integers.  p_corp: back-off
+ * query of M_n in descending n with the last n tokens; p_prompt: the same construction
+ * over the sequence's own committed tokens (no pruning).  Drafts already produced in this
+ * call extend the query suffix only.  A component with zero weight or without a match at
+ * any order takes no part; if neither does, the draft is the most frequent corpus token.
+ *
+ *   tokens   device, int32[B][stride]: committed tokens of each sequence
+ *   len      device, int32[B]: committed length L_b (1 <= L_b <= stride)
+ *   drafts   device, int32[B][k] (written)
+ *   k        1..TASC_MAX_ROWS-1;  0 <= lambda_num <= lambda_den <= 256
+ * Asynchronous on the stream.  Errors: EINVAL (also when stride is too large for the
+ * kernel's shared-memory successor table: stride <= 12288).
+ */
+tasc_status tasc_draft(const tasc_drafter* d, const int32_t* tokens, int64_t stride, const int32_t* len,
+                       int32_t B, int32_t k, int32_t lambda_num, int32_t lambda_den, int32_t* drafts,
+                       tasc_stream stream);
+
+/* -------------------------------------------------------------------- model */
+
+/* Decoder shape (pre-norm, RMSNorm, rotate-half RoPE, grouped-query attention, SwiGLU, no biases). */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+    int32_t dtype;          /* TASC_F32 or TASC_BF16: type of weight matrices, KV pool and GEMM inputs */
+    float   rope_base;      /* e.g. 10000 */
+    float   rms_eps;        /* e.g. 1e-6 */
+    int32_t max_positions;  /* size of the rotary table: every position must be < max_positions */
+    int32_t page_size;      /* tokens per KV page (16) */
+} tasc_model_desc;
+
+/*
+ * Device pointers to the weights, borrowed for the lifetime of the model handle.
+ * Matrices are row-major [out_features][in_features] in the model dtype; norm gains are float32.
+ * The per-layer members are HOST arrays of n_layers device pointers.
+ */
+typedef struct {
+    const void*  embed;          /* [vocab][d_model] */
+    const void*  lm_head;        /* [vocab][d_model] (may equal embed) */
+    const float* final_norm;     /* [d_model] */
+    const float* const* attn_norm;   /* each [d_model] */
+    const void*  const* wqkv;        /* each [(n_q + 2 n_kv) * head_dim][d_model]: q heads, k heads, v heads */
+    const void*  const* wo;          /* each [d_model][n_q * head_dim] */
+    const float* const* mlp_norm;    /* each [d_model] */
+    const void*  const* w_gate_up;   /* each [2 * d_ff][d_model]: gate rows, then up rows */
+    const void*  const* w_down;      /* each [d_model][d_ff] */
+} tasc_weights;
+
+/*
+ * Paged KV cache, caller-owned.  pool layout (model dtype):
+ *   [n_layers][2 (K, V)][n_pages][n_kv_heads][page_size][head_dim]
+ * block_table[b][j] is the page holding positions j*page_size .. of sequence b.
+ */
+typedef struct {
+    void*          pool;               /* device */
+    int64_t        n_pages;
+    const int32_t* block_table;        /* device, int32[B][max_pages_per_seq], every id in [0, n_pages) */
+    int32_t        max_pages_per_seq;
+} tasc_kv;
+
+/*
+ * Committed tokens of the batch.  The KV cache of sequence b holds positions 0 .. len[b]-2:
+ * the last committed token has not been through the model yet.
+ */
+typedef struct {
+    int32_t*       tokens;     /* device, int32[B][stride] */
+    int64_t        stride;
+    int32_t*       len;        /* device, int32[B] */
+    const int32_t* stop_len;   /* device, int32[B] or NULL: a sequence with len >= stop_len is skipped */
+} tasc_seqs;
+
+/* Validates the shape, builds the rotary table and the weight tensor maps.  Errors: EINVAL, ENOMEM, ECUDA. */
+tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc_weights* weights, tasc_model** out);
+tasc_status tasc_model_destroy(tasc_model* m);
+
+/* Bytes of workspace that step calls need for up to B_max sequences and k_max drafts. */
+size_t tasc_workspace_bytes(const tasc_model* m, int32_t B_max, int32_t k_max);
+
+/*
+ * Run the committed tokens 0 .. len[b]-2 of every sequence through the model to fill the KV
+ * cache (no logits).  max_len (host value) >= every len[b]; it fixes the number of chunks.
+ * Asynchronous.  Errors: EINVAL.
+ */
+tasc_status tasc_prefill(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, int32_t B, int32_t max_len,
+                         void* workspace, size_t workspace_bytes, tasc_stream stream);
+
+/*
+ * One verification step (Section 5.1: the target model verifies the drafted tokens in a single
+ * forward pass and a prefix is accepted; greedy acceptance, i.e. beam size 1).
+ * Rows [last committed token, d_1..d_k] of sequence b run at positions L-1 .. L-1+k (L = len[b]);
+ * their K/V are appended to the cache; y_i = argmax of row i's logits (smallest id on ties);
+ * a = longest prefix with d_j = y_{j-1}; d_1..d_a and y_a are appended to tokens and len grows by
+ * a+1, which also rolls the KV cache back over the rejected rows.
+ *
+ *   drafts         device, int32[B][k]
+ *   forced_targets device, int32[B][k+1] or NULL: replaces y in the accept rule and in what is
+ *                  committed (teacher-forced mode); the forward pass still runs in full
+ *   n_accepted     device, int32[B] (written): a, 0..k
+ *   next_token     device, int32[B] (written): the token committed after the accepted drafts
+ *   target_tokens  device, int32[B][k+1] or NULL (written): y
+ *   logits_dbg     device, float[B][k+1][vocab] or NULL (written): all logits (debug; large)
+ * Asynchronous.  Errors: EINVAL (k+1 > TASC_MAX_ROWS, workspace too small, ...).
+ */
+tasc_status tasc_verify_step(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, const int32_t* drafts,
+                             int32_t B, int32_t k, const int32_t* forced_targets,
+                             int32_t* n_accepted, int32_t* next_token, int32_t* target_tokens, float* logits_dbg,
+                             void* workspace, size_t workspace_bytes, tasc_stream stream);
+
+/* How tasc_generate chooses the targets of each step. */
+#define TASC_MODE_GREEDY        0   /* targets = the model's own argmax */
+#define TASC_MODE_CONTINUATION  1   /* teacher-forced: targets = continuation[b][g .. g+k], g = tokens generated so far */
+#define TASC_MODE_FORCED_ACCEPT 2   /* teacher-forced: exactly forced_accept drafts are accepted every step */
+
+typedef struct {
+    int32_t k;
+    int32_t lambda_num, lambda_den;
+    int32_t mode;
+    int32_t forced_accept;              /* TASC_MODE_FORCED_ACCEPT: 0..k */
+    const int32_t* continuation;        /* TASC_MODE_CONTINUATION: device, int32[B][continuation_stride] */
+    int64_t continuation_stride;        /* >= max_new + k + 1 */
+} tasc_draft_params;
+
+typedef struct {
+    int64_t steps;                      /* speculative steps enqueued */
+    int64_t committed;                  /* tokens committed over all sequences (before truncation to max_new) */
+    int64_t accepted_hist[TASC_MAX_ROWS]; /* accepted_hist[a] = sequence-steps that accepted exactly a drafts */
+    float   prefill_ms, decode_ms;      /* device time of the two phases */
+} tasc_stats;
+
+/*
+ * Prefill, then repeat [draft k tokens -> verify step] until every sequence has generated max_new
+ * tokens.  On entry seqs holds the prompts (len = prompt lengths, stride >= prompt + max_new + k + 1);
+ * on return tokens/len hold prompt + generated tokens (a sequence may overshoot max_new by up to k).
+ *   out    device, int32[B][max_new] (written): the first max_new generated tokens
+ *   stats  host (written), may be NULL
+ * Synchronises the stream.  Errors: EINVAL, ECUDA, and device-side statuses (ENOKV, ETIMEOUT).
+ */
+tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* d, const tasc_kv* kv, const tasc_seqs* seqs,
+                          int32_t B, int32_t max_new, const tasc_draft_params* params, int32_t* out,
+                          tasc_stats* stats, void* workspace, size_t workspace_bytes, tasc_stream stream);
+
+/* Synchronise the stream and return the device status word of the workspace (TASC_OK if clean); clears it. */
+tasc_status tasc_poll_status(void* workspace, tasc_stream stream);
+
+/*
+ * Y[M][N] (float32) = X[M][K] * W[N][K]^T for bf16 X and W on the tensor cores, the building block of
+ * every projection of the verify forward (exported for unit tests and profiling).
+ *   x, w       device, bf16, row-major, 16-byte aligned; K a multiple of 8
+ *   y          device, float32[M][N]
+ *   workspace  device, at least tasc_gemm_workspace_bytes(M, N, K) bytes (split-K partial sums)
+ * Asynchronous.  Errors: EINVAL, ECUDA.
+ */
+tasc_status tasc_gemm_bf16(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                           void* workspace, size_t workspace_bytes, tasc_stream stream);
+size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
+
+const char* tasc_status_string(tasc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TASC_H */

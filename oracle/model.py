@@ -126,3 +126,8 @@ def argmax_and_gap(logits):
         return idx, np.full(idx.shape, np.inf)
     top2 = np.partition(logits, -2, axis=-1)[..., -2:]
     return idx, (top2[..., 1] - top2[..., 0]).astype(np.float64)
+
+
+def linear(x, w):
+    """y = x W^T for row-major W [out_features, in_features] (the projection every layer uses)."""
+    return x @ w.T

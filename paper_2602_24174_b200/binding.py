@@ -1,0 +1,288 @@
+"""ctypes binding of libtasc.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in ``include/tasc.h``; tensors are
+torch CUDA tensors used as device buffers, and every step of the path runs inside the library's
+kernels.  Importing this module fails loudly if the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtasc.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2602_24174_b200.build` "
+        "(there is no CPU or PyTorch fallback for this path)")
+
+lib = C.CDLL(LIB_PATH)
+
+OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ENOKV, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+MAX_ORDER, MAX_ROWS, VOCAB_BITS = 5, 16, 20
+F32, BF16 = 0, 1
+MODE_GREEDY, MODE_CONTINUATION, MODE_FORCED_ACCEPT = 0, 1, 2
+
+
+class TascError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib.tasc_status_string(code).decode()} ({code})")
+
+
+class NgramEntry(C.Structure):
+    _fields_ = [("n", C.c_int32), ("ctx", C.c_int32 * MAX_ORDER), ("next", C.c_int32), ("count", C.c_uint32)]
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32), ("dtype", C.c_int32),
+                ("rope_base", C.c_float), ("rms_eps", C.c_float), ("max_positions", C.c_int32), ("page_size", C.c_int32)]
+
+
+class Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+                ("attn_norm", C.POINTER(C.c_void_p)), ("wqkv", C.POINTER(C.c_void_p)), ("wo", C.POINTER(C.c_void_p)),
+                ("mlp_norm", C.POINTER(C.c_void_p)), ("w_gate_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p))]
+
+
+class Kv(C.Structure):
+    _fields_ = [("pool", C.c_void_p), ("n_pages", C.c_int64), ("block_table", C.c_void_p), ("max_pages_per_seq", C.c_int32)]
+
+
+class Seqs(C.Structure):
+    _fields_ = [("tokens", C.c_void_p), ("stride", C.c_int64), ("len", C.c_void_p), ("stop_len", C.c_void_p)]
+
+
+class DraftParams(C.Structure):
+    _fields_ = [("k", C.c_int32), ("lambda_num", C.c_int32), ("lambda_den", C.c_int32), ("mode", C.c_int32),
+                ("forced_accept", C.c_int32), ("continuation", C.c_void_p), ("continuation_stride", C.c_int64)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("steps", C.c_int64), ("committed", C.c_int64), ("accepted_hist", C.c_int64 * MAX_ROWS),
+                ("prefill_ms", C.c_float), ("decode_ms", C.c_float)]
+
+
+_P = C.c_void_p
+lib.tasc_status_string.restype = C.c_char_p
+lib.tasc_status_string.argtypes = [C.c_int32]
+lib.tasc_drafter_build.argtypes = [_P, _P, C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(_P)]
+lib.tasc_drafter_export.argtypes = [_P, C.POINTER(NgramEntry), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
+lib.tasc_drafter_destroy.argtypes = [_P]
+lib.tasc_draft.argtypes = [_P, _P, C.c_int64, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P]
+lib.tasc_model_create.argtypes = [C.POINTER(ModelDesc), C.POINTER(Weights), C.POINTER(_P)]
+lib.tasc_model_destroy.argtypes = [_P]
+lib.tasc_workspace_bytes.restype = C.c_size_t
+lib.tasc_workspace_bytes.argtypes = [_P, C.c_int32, C.c_int32]
+lib.tasc_prefill.argtypes = [_P, C.POINTER(Kv), C.POINTER(Seqs), C.c_int32, C.c_int32, _P, C.c_size_t, _P]
+lib.tasc_verify_step.argtypes = [_P, C.POINTER(Kv), C.POINTER(Seqs), _P, C.c_int32, C.c_int32, _P, _P, _P, _P, _P, _P,
+                                 C.c_size_t, _P]
+lib.tasc_generate.argtypes = [_P, _P, C.POINTER(Kv), C.POINTER(Seqs), C.c_int32, C.c_int32, C.POINTER(DraftParams), _P,
+                              C.POINTER(Stats), _P, C.c_size_t, _P]
+lib.tasc_poll_status.argtypes = [_P, _P]
+lib.tasc_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
+lib.tasc_gemm_workspace_bytes.restype = C.c_size_t
+lib.tasc_gemm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+for _f in ("tasc_drafter_build", "tasc_drafter_export", "tasc_drafter_destroy", "tasc_draft", "tasc_model_create",
+           "tasc_model_destroy", "tasc_prefill", "tasc_verify_step", "tasc_generate", "tasc_poll_status", "tasc_gemm_bf16"):
+    getattr(lib, _f).restype = C.c_int32
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise TascError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype) -> torch.Tensor:
+    assert t.is_cuda and t.dtype == dtype and t.is_contiguous(), (t.device, t.dtype, t.is_contiguous())
+    return t
+
+
+class Drafter:
+    """tasc_drafter handle: corpus n-gram tables on the device."""
+
+    def __init__(self, handle, n_max: int):
+        self._h, self.n_max = handle, n_max
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib.tasc_drafter_destroy(self._h)
+            self._h = None
+
+    def export(self):
+        """(entries as int64[E, MAX_ORDER + 3] rows (n, ctx padded with -1, next, count), fallback token)."""
+        n = C.c_int64(0)
+        fb = C.c_int32(0)
+        _check(lib.tasc_drafter_export(self._h, None, 0, C.byref(n), C.byref(fb)), "tasc_drafter_export")
+        buf = (NgramEntry * max(n.value, 1))()
+        _check(lib.tasc_drafter_export(self._h, buf, n.value, C.byref(n), C.byref(fb)), "tasc_drafter_export")
+        raw = np.frombuffer(buf, dtype=np.int32).reshape(-1, MAX_ORDER + 3)[:n.value]
+        out = raw.astype(np.int64)
+        out[:, MAX_ORDER + 2] = raw[:, MAX_ORDER + 2].view(np.uint32)
+        return out, fb.value
+
+
+def tasc_drafter_build(corpus_tokens: torch.Tensor, doc_offsets: torch.Tensor, n_max: int, p_min: int, vocab: int) -> Drafter:
+    _dev(corpus_tokens, torch.int32)
+    _dev(doc_offsets, torch.int64)
+    h = _P()
+    _check(lib.tasc_drafter_build(_ptr(corpus_tokens), _ptr(doc_offsets), doc_offsets.numel() - 1, n_max, p_min, vocab,
+                                  _stream(), C.byref(h)), "tasc_drafter_build")
+    return Drafter(h, n_max)
+
+
+def tasc_draft(drafter: Drafter, tokens: torch.Tensor, length: torch.Tensor, k: int, lambda_num: int = 3,
+               lambda_den: int = 4, out: torch.Tensor | None = None) -> torch.Tensor:
+    _dev(tokens, torch.int32)
+    _dev(length, torch.int32)
+    B, stride = tokens.shape
+    if out is None:
+        out = torch.empty((B, k), dtype=torch.int32, device=tokens.device)
+    _check(lib.tasc_draft(drafter._h, _ptr(tokens), stride, _ptr(length), B, k, lambda_num, lambda_den, _ptr(out), _stream()),
+           "tasc_draft")
+    return out
+
+
+_TORCH_DTYPE = {F32: torch.float32, BF16: torch.bfloat16}
+
+
+class Model:
+    """tasc_model handle plus the device buffers it borrows (kept alive here)."""
+
+    def __init__(self, shape, weights: dict, max_positions: int, page_size: int = 16):
+        """``shape``: object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab, dtype ("f32"/"bf16"),
+        rope_base, rms_eps.  ``weights``: dict of CUDA tensors laid out as the C header describes."""
+        self.shape = shape
+        self.dtype = F32 if shape.dtype == "f32" else BF16
+        self.tdtype = _TORCH_DTYPE[self.dtype]
+        self.page_size = page_size
+        self.max_positions = max_positions
+        L = shape.n_layers
+        self._keep = weights
+        desc = ModelDesc(L, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ff, shape.vocab,
+                         self.dtype, shape.rope_base, shape.rms_eps, max_positions, page_size)
+
+        def arr(name, dtype):
+            a = (C.c_void_p * L)()
+            for l in range(L):
+                a[l] = _dev(weights["layers"][l][name], dtype).data_ptr()
+            return a
+
+        self._arrays = [arr("attn_norm", torch.float32), arr("wqkv", self.tdtype), arr("wo", self.tdtype),
+                        arr("mlp_norm", torch.float32), arr("w_gate_up", self.tdtype), arr("w_down", self.tdtype)]
+        w = Weights(_dev(weights["embed"], self.tdtype).data_ptr(), _dev(weights["lm_head"], self.tdtype).data_ptr(),
+                    _dev(weights["final_norm"], torch.float32).data_ptr(), *[C.cast(a, C.POINTER(C.c_void_p)) for a in self._arrays])
+        h = _P()
+        _check(lib.tasc_model_create(C.byref(desc), C.byref(w), C.byref(h)), "tasc_model_create")
+        self._h = h
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib.tasc_model_destroy(self._h)
+            self._h = None
+
+    def workspace_bytes(self, B: int, k: int) -> int:
+        n = lib.tasc_workspace_bytes(self._h, B, k)
+        if n == 0:
+            raise TascError(EINVAL, "tasc_workspace_bytes")
+        return n
+
+    def new_workspace(self, B: int, k: int, device="cuda") -> torch.Tensor:
+        return torch.zeros(self.workspace_bytes(B, k), dtype=torch.uint8, device=device)
+
+    def new_kv(self, B: int, max_len: int, device="cuda"):
+        """A KV pool with one private run of pages per sequence: (pool, block_table, Kv struct)."""
+        s = self.shape
+        pages_per_seq = -(-max_len // self.page_size)
+        n_pages = B * pages_per_seq
+        pool = torch.zeros((s.n_layers, 2, n_pages, s.n_kv_heads, self.page_size, s.head_dim), dtype=self.tdtype, device=device)
+        # pages of a sequence are deliberately not contiguous in the pool: page j of sequence b is j * B + b
+        bt = (torch.arange(pages_per_seq, dtype=torch.int32)[None, :] * B + torch.arange(B, dtype=torch.int32)[:, None])
+        bt = bt.contiguous().to(device)
+        return pool, bt, Kv(pool.data_ptr(), n_pages, bt.data_ptr(), pages_per_seq)
+
+
+def make_seqs(tokens: torch.Tensor, length: torch.Tensor, stop_len: torch.Tensor | None = None) -> Seqs:
+    _dev(tokens, torch.int32)
+    _dev(length, torch.int32)
+    return Seqs(tokens.data_ptr(), tokens.shape[1], length.data_ptr(), None if stop_len is None else _dev(stop_len, torch.int32).data_ptr())
+
+
+def tasc_prefill(model: Model, kv: Kv, seqs: Seqs, B: int, max_len: int, workspace: torch.Tensor):
+    _check(lib.tasc_prefill(model._h, C.byref(kv), C.byref(seqs), B, max_len, _ptr(workspace), workspace.numel(), _stream()),
+           "tasc_prefill")
+
+
+def tasc_verify_step(model: Model, kv: Kv, seqs: Seqs, drafts: torch.Tensor, workspace: torch.Tensor, *,
+                     forced_targets: torch.Tensor | None = None, want_targets: bool = False, want_logits: bool = False):
+    """Returns (n_accepted[B], next_token[B], target_tokens[B, k+1] or None, logits[B, k+1, V] or None)."""
+    _dev(drafts, torch.int32)
+    B, k = drafts.shape
+    dev = drafts.device
+    n_acc = torch.empty(B, dtype=torch.int32, device=dev)
+    nxt = torch.empty(B, dtype=torch.int32, device=dev)
+    tgt = torch.empty((B, k + 1), dtype=torch.int32, device=dev) if want_targets else None
+    logits = torch.empty((B, k + 1, model.shape.vocab), dtype=torch.float32, device=dev) if want_logits else None
+    if forced_targets is not None:
+        _dev(forced_targets, torch.int32)
+    _check(lib.tasc_verify_step(model._h, C.byref(kv), C.byref(seqs), _ptr(drafts), B, k, _ptr(forced_targets), _ptr(n_acc),
+                                _ptr(nxt), _ptr(tgt), _ptr(logits), _ptr(workspace), workspace.numel(), _stream()),
+           "tasc_verify_step")
+    return n_acc, nxt, tgt, logits
+
+
+def tasc_generate(model: Model, drafter: Drafter, kv: Kv, seqs: Seqs, B: int, max_new: int, k: int, workspace: torch.Tensor, *,
+                  lambda_num: int = 3, lambda_den: int = 4, mode: int = MODE_GREEDY, forced_accept: int = 0,
+                  continuation: torch.Tensor | None = None, out: torch.Tensor | None = None):
+    """Returns (out[B, max_new] int32 CUDA tensor, Stats)."""
+    if out is None:
+        out = torch.empty((B, max_new), dtype=torch.int32, device=workspace.device)
+    p = DraftParams(k, lambda_num, lambda_den, mode, forced_accept,
+                    None if continuation is None else _dev(continuation, torch.int32).data_ptr(),
+                    0 if continuation is None else continuation.shape[1])
+    st = Stats()
+    _check(lib.tasc_generate(model._h, drafter._h, C.byref(kv), C.byref(seqs), B, max_new, C.byref(p), _ptr(out), C.byref(st),
+                             _ptr(workspace), workspace.numel(), _stream()), "tasc_generate")
+    return out, st
+
+
+def tasc_poll_status(workspace: torch.Tensor):
+    _check(lib.tasc_poll_status(_ptr(workspace), _stream()), "tasc_poll_status")
+
+
+def tasc_gemm_bf16(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
+    """Y[M, N] float32 = X[M, K] @ W[N, K]^T for bf16 CUDA tensors."""
+    _dev(x, torch.bfloat16)
+    _dev(w, torch.bfloat16)
+    M, K = x.shape
+    N = w.shape[0]
+    nbytes = lib.tasc_gemm_workspace_bytes(M, N, K)
+    ws = torch.zeros(max(nbytes, 256), dtype=torch.uint8, device=x.device)
+    y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    _check(lib.tasc_gemm_bf16(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(ws), ws.numel(), _stream()), "tasc_gemm_bf16")
+    tasc_poll_status(ws)
+    return y
+
+
+def weights_to_device(w: dict, dtype: str, device="cuda") -> dict:
+    """Host float32 weight dict (as produced by the workload generator) -> CUDA tensors in the model dtype."""
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    conv = lambda a, t: torch.from_numpy(np.ascontiguousarray(a)).to(device=device, dtype=t).contiguous()
+    out = {"embed": conv(w["embed"], td), "final_norm": conv(w["final_norm"], torch.float32), "layers": []}
+    out["lm_head"] = out["embed"] if w["lm_head"] is w["embed"] else conv(w["lm_head"], td)
+    for lw in w["layers"]:
+        out["layers"].append({k: conv(v, torch.float32 if k.endswith("norm") else td) for k, v in lw.items()})
+    return out

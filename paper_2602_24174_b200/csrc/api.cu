@@ -1,0 +1,445 @@
+// C-ABI layer: model handle, workspace layout, the verify forward as a sequence of kernel launches,
+// prefill, the speculative step and the generation loop.  Argument checking and launch order only;
+// all arithmetic is in the kernel files.
+#include "kernels.h"
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+struct tasc_model {
+    tasc_model_desc desc;
+    const void* embed;
+    const void* lm_head;
+    const float* final_norm;
+    std::vector<const float*> attn_norm, mlp_norm;
+    std::vector<const void*> wqkv, wo, w_gate_up, w_down;
+    float2* rope;                                   // [max_positions][head_dim / 2] (cos, sin), library-owned
+    // tensor maps of the weight matrices (bf16 models): box = 64 x 128
+    std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
+    CUtensorMap tm_lm;
+    int qkv_rows, q_dim, kv_dim;
+};
+
+namespace tasc {
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr size_t MIN_PARTIAL_BYTES = 64ull << 20;
+
+struct Layout {
+    size_t off = 0;
+    template <typename U> U* take(uint8_t* base, size_t count) {
+        U* p = reinterpret_cast<U*>(base + off);
+        off += (count * sizeof(U) + ALIGN - 1) / ALIGN * ALIGN;
+        return p;
+    }
+};
+
+struct Workspace {
+    int* status;
+    long long* hist;              // [TASC_MAX_ROWS]
+    int* min_gen;
+    RowPlan rp;
+    unsigned long long* argmax;   // [M]
+    int32_t *drafts, *targets, *n_accepted, *next_token, *prompt_len, *stop_len;
+    float* x;                     // [M][d] residual stream
+    void *h, *q, *o, *act;        // model dtype
+    float* partials;
+    size_t partial_bytes;
+    float* att_scratch;
+    size_t bytes;
+};
+
+// The layout is always made for TASC_MAX_ROWS rows per sequence so that every call agrees on it.
+Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
+    const tasc_model_desc& d = m->desc;
+    uint8_t* base = static_cast<uint8_t*>(base_);
+    const size_t M = (size_t)B * TASC_MAX_ROWS;
+    const size_t esz = d.dtype == TASC_F32 ? 4 : 2;
+    Layout L;
+    Workspace w;
+    w.status = L.take<int>(base, 64);
+    w.hist = L.take<long long>(base, TASC_MAX_ROWS);
+    w.min_gen = L.take<int>(base, 64);
+    w.rp.row_tok = L.take<int>(base, M);
+    w.rp.row_pos = L.take<int>(base, M);
+    w.rp.seq_pos0 = L.take<int>(base, B);
+    w.rp.seq_rows = L.take<int>(base, B);
+    w.argmax = L.take<unsigned long long>(base, M);
+    w.drafts = L.take<int32_t>(base, M);
+    w.targets = L.take<int32_t>(base, M);
+    w.n_accepted = L.take<int32_t>(base, B);
+    w.next_token = L.take<int32_t>(base, B);
+    w.prompt_len = L.take<int32_t>(base, B);
+    w.stop_len = L.take<int32_t>(base, B);
+    w.x = L.take<float>(base, M * d.d_model);
+    w.h = L.take<uint8_t>(base, M * d.d_model * esz);
+    w.q = L.take<uint8_t>(base, M * m->q_dim * esz);
+    w.o = L.take<uint8_t>(base, M * m->q_dim * esz);
+    w.act = L.take<uint8_t>(base, M * d.d_ff * esz);
+    const size_t n_max = std::max<size_t>({(size_t)m->qkv_rows, (size_t)2 * d.d_ff, (size_t)d.d_model});
+    w.partial_bytes = std::max(MIN_PARTIAL_BYTES, M * n_max * sizeof(float));
+    w.partials = L.take<float>(base, w.partial_bytes / sizeof(float));
+    const int splits_max = attention_splits(B, d.n_kv_heads, 1 << 30);
+    w.att_scratch = L.take<float>(base, attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max) / sizeof(float));
+    w.bytes = L.off;
+    return w;
+}
+
+__global__ void init_generate_kernel(const int32_t* len, int32_t* prompt_len, int32_t* stop_len, int B, int max_new) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    prompt_len[b] = len[b];
+    stop_len[b] = len[b] + max_new;
+}
+
+struct KvView {
+    void* k; void* v;
+};
+KvView layer_kv(const tasc_model* m, const tasc_kv* kv, int layer) {
+    const tasc_model_desc& d = m->desc;
+    const size_t esz = d.dtype == TASC_F32 ? 4 : 2;
+    const size_t per = (size_t)kv->n_pages * d.n_kv_heads * d.page_size * d.head_dim * esz;
+    uint8_t* base = static_cast<uint8_t*>(kv->pool) + (size_t)layer * 2 * per;
+    return KvView{base, base + per};
+}
+
+// One GEMM of the forward: P = X[M][K] * W[N][K]^T as split partials; returns the number of splits.
+template <typename T>
+tasc_status run_gemm(const tasc_model* m, const Workspace& w, const void* X, const CUtensorMap* tmX, const void* W,
+                     const CUtensorMap* tmW, int M, int N, int K, int* splits, unsigned long long* argmax, float* logits,
+                     cudaStream_t s) {
+    if constexpr (sizeof(T) == 4) {
+        (void)m; (void)tmX; (void)tmW;
+        launch_gemm_f32(static_cast<const float*>(X), static_cast<const float*>(W), w.partials, M, N, K, argmax, logits, s);
+        *splits = 1;
+        return TASC_OK;
+    } else {
+        (void)X; (void)W;
+        GemmPlan plan = plan_gemm(M, N, K, w.partial_bytes);
+        if (argmax) plan.splits = 1;
+        *splits = plan.splits;
+        return launch_gemm_bf16(tmW, tmX, w.partials, M, N, K, plan, argmax, logits, w.status, s);
+    }
+}
+
+// Forward of M = B * R rows described by w.rp; fills the KV cache; optionally the LM head + argmax.
+template <typename T>
+tasc_status forward(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
+                    cudaStream_t s) {
+    const tasc_model_desc& d = m->desc;
+    const int M = B * R;
+    const int max_ctx = kv->max_pages_per_seq * d.page_size;
+    const int att_splits = attention_splits(B, d.n_kv_heads, max_ctx);
+    CUtensorMap tm_h, tm_o, tm_act;
+    if constexpr (sizeof(T) == 2) {
+        const GemmPlan p = plan_gemm(M, d.d_model, d.d_model, w.partial_bytes);      // BN depends on M only
+        tasc_status st;
+        if ((st = encode_tmap_bf16(&tm_h, w.h, M, d.d_model, p.BN)) != TASC_OK) return st;
+        if ((st = encode_tmap_bf16(&tm_o, w.o, M, m->q_dim, p.BN)) != TASC_OK) return st;
+        if ((st = encode_tmap_bf16(&tm_act, w.act, M, d.d_ff, p.BN)) != TASC_OK) return st;
+    }
+    T* h = static_cast<T*>(w.h);
+    T* q = static_cast<T*>(w.q);
+    T* o = static_cast<T*>(w.o);
+    T* act = static_cast<T*>(w.act);
+    launch_embed_norm<T>(static_cast<const T*>(m->embed), w.rp.row_tok, m->attn_norm[0], d.rms_eps, w.x, h, M, d.d_model, s);
+    for (int l = 0; l < d.n_layers; ++l) {
+        const KvView kvl = layer_kv(m, kv, l);
+        int sp = 1;
+        tasc_status st;
+        const bool bf = sizeof(T) == 2;
+        st = run_gemm<T>(m, w, h, &tm_h, m->wqkv[l], bf ? &m->tm_qkv[l] : nullptr, M, m->qkv_rows, d.d_model, &sp, nullptr, nullptr, s);
+        if (st != TASC_OK) return st;
+        launch_qkv_rope_append<T>(w.partials, sp, w.rp, m->rope, q, static_cast<T*>(kvl.k), static_cast<T*>(kvl.v),
+                                  kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, M, R, d.n_q_heads,
+                                  d.n_kv_heads, d.head_dim, d.max_positions, w.status, s);
+        launch_attention<T>(q, static_cast<const T*>(kvl.k), static_cast<const T*>(kvl.v), kv->block_table,
+                            kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, w.att_scratch, B, R, d.n_q_heads,
+                            d.n_kv_heads, d.head_dim, att_splits, s);
+        st = run_gemm<T>(m, w, o, &tm_o, m->wo[l], bf ? &m->tm_o[l] : nullptr, M, d.d_model, m->q_dim, &sp, nullptr, nullptr, s);
+        if (st != TASC_OK) return st;
+        launch_residual_norm<T>(w.partials, sp, w.x, m->mlp_norm[l], d.rms_eps, h, M, d.d_model, s);
+        st = run_gemm<T>(m, w, h, &tm_h, m->w_gate_up[l], bf ? &m->tm_gu[l] : nullptr, M, 2 * d.d_ff, d.d_model, &sp, nullptr, nullptr, s);
+        if (st != TASC_OK) return st;
+        launch_silu_mul<T>(w.partials, sp, act, M, d.d_ff, s);
+        st = run_gemm<T>(m, w, act, &tm_act, m->w_down[l], bf ? &m->tm_down[l] : nullptr, M, d.d_model, d.d_ff, &sp, nullptr, nullptr, s);
+        if (st != TASC_OK) return st;
+        const float* next_gain = l + 1 < d.n_layers ? m->attn_norm[l + 1] : m->final_norm;
+        launch_residual_norm<T>(w.partials, sp, w.x, next_gain, d.rms_eps, h, M, d.d_model, s);
+    }
+    if (lm_head) {
+        int sp = 1;
+        launch_fill_u64(w.argmax, 0ull, M, s);
+        tasc_status st = run_gemm<T>(m, w, h, &tm_h, m->lm_head, sizeof(T) == 2 ? &m->tm_lm : nullptr, M, d.vocab, d.d_model,
+                                     &sp, w.argmax, logits, s);
+        if (st != TASC_OK) return st;
+    }
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
+tasc_status forward_any(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
+                        cudaStream_t s) {
+    return m->desc.dtype == TASC_F32 ? forward<float>(m, kv, w, B, R, lm_head, logits, s)
+                                     : forward<__nv_bfloat16>(m, kv, w, B, R, lm_head, logits, s);
+}
+
+bool check_common(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, int B, void* ws, size_t ws_bytes) {
+    if (!m || !kv || !seqs || !ws || B < 1) return false;
+    if (!kv->pool || !kv->block_table || kv->n_pages < 1 || kv->max_pages_per_seq < 1) return false;
+    if (!seqs->tokens || !seqs->len || seqs->stride < 1) return false;
+    if (reinterpret_cast<uintptr_t>(ws) % ALIGN) return false;
+    return ws_bytes >= layout_workspace(m, B, ws).bytes;
+}
+
+tasc_status verify_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, const Workspace& w,
+                           const int32_t* drafts, int B, int k, const int32_t* forced, int32_t* n_accepted,
+                           int32_t* next_token, int32_t* target_tokens, float* logits, cudaStream_t s) {
+    const int R = k + 1;
+    launch_rows_verify(w.rp, seqs->tokens, seqs->stride, seqs->len, seqs->stop_len, drafts, B, R, m->desc.vocab, w.status, s);
+    tasc_status st = forward_any(m, kv, w, B, R, true, logits, s);
+    if (st != TASC_OK) return st;
+    launch_accept(w.argmax, w.rp, drafts, forced, seqs->tokens, seqs->stride, seqs->len, B, R, n_accepted, next_token,
+                  target_tokens, w.hist, s);
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
+tasc_status prefill_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, const Workspace& w, int B,
+                            int max_len, cudaStream_t s) {
+    const int R = TASC_MAX_ROWS;
+    const int chunks = (std::max(max_len - 1, 0) + R - 1) / R;
+    for (int c = 0; c < chunks; ++c) {
+        launch_rows_prefill(w.rp, seqs->tokens, seqs->stride, seqs->len, B, R, c, m->desc.vocab, w.status, s);
+        tasc_status st = forward_any(m, kv, w, B, R, false, nullptr, s);
+        if (st != TASC_OK) return st;
+    }
+    return TASC_OK;
+}
+
+}  // namespace
+}  // namespace tasc
+
+using namespace tasc;
+
+extern "C" tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc_weights* wt, tasc_model** out) {
+    if (!out) return TASC_EINVAL;
+    *out = nullptr;
+    if (!desc || !wt) return TASC_EINVAL;
+    const tasc_model_desc& d = *desc;
+    if (d.n_layers < 1 || d.d_model < 8 || d.n_q_heads < 1 || d.n_kv_heads < 1 || d.n_q_heads % d.n_kv_heads ||
+        d.head_dim < 8 || d.head_dim > 256 || d.head_dim % 8 || d.d_ff < 8 || d.vocab < 2 ||
+        d.vocab > (1 << TASC_VOCAB_BITS) || (d.dtype != TASC_F32 && d.dtype != TASC_BF16) || d.max_positions < 1 ||
+        d.page_size < 1 || d.d_model % 8 || d.d_ff % 8 || !(d.rope_base > 0.f) || !(d.rms_eps >= 0.f))
+        return TASC_EINVAL;
+    if (!wt->embed || !wt->lm_head || !wt->final_norm || !wt->attn_norm || !wt->wqkv || !wt->wo || !wt->mlp_norm ||
+        !wt->w_gate_up || !wt->w_down)
+        return TASC_EINVAL;
+    tasc_model* m = new (std::nothrow) tasc_model();
+    if (!m) return TASC_ENOMEM;
+    m->desc = d;
+    m->embed = wt->embed; m->lm_head = wt->lm_head; m->final_norm = wt->final_norm;
+    m->q_dim = d.n_q_heads * d.head_dim;
+    m->kv_dim = d.n_kv_heads * d.head_dim;
+    m->qkv_rows = m->q_dim + 2 * m->kv_dim;
+    m->rope = nullptr;
+    for (int l = 0; l < d.n_layers; ++l) {
+        if (!wt->attn_norm[l] || !wt->wqkv[l] || !wt->wo[l] || !wt->mlp_norm[l] || !wt->w_gate_up[l] || !wt->w_down[l]) {
+            delete m;
+            return TASC_EINVAL;
+        }
+        m->attn_norm.push_back(wt->attn_norm[l]); m->mlp_norm.push_back(wt->mlp_norm[l]);
+        m->wqkv.push_back(wt->wqkv[l]); m->wo.push_back(wt->wo[l]);
+        m->w_gate_up.push_back(wt->w_gate_up[l]); m->w_down.push_back(wt->w_down[l]);
+    }
+    tasc_status st = TASC_OK;
+    if (d.dtype == TASC_BF16) {
+        m->tm_qkv.resize(d.n_layers); m->tm_o.resize(d.n_layers); m->tm_gu.resize(d.n_layers); m->tm_down.resize(d.n_layers);
+        st = gemm_set_attributes();
+        for (int l = 0; l < d.n_layers && st == TASC_OK; ++l) {
+            st = encode_tmap_bf16(&m->tm_qkv[l], m->wqkv[l], m->qkv_rows, d.d_model, 128);
+            if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_o[l], m->wo[l], d.d_model, m->q_dim, 128);
+            if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_gu[l], m->w_gate_up[l], 2 * (uint64_t)d.d_ff, d.d_model, 128);
+            if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_down[l], m->w_down[l], d.d_model, d.d_ff, 128);
+        }
+        if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_lm, m->lm_head, d.vocab, d.d_model, 128);
+    }
+    if (st == TASC_OK) {
+        const size_t n = (size_t)d.max_positions * (d.head_dim / 2);
+        if (cudaMalloc(reinterpret_cast<void**>(&m->rope), n * sizeof(float2)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            st = TASC_ENOMEM;
+        } else {
+            launch_rope_table(m->rope, d.max_positions, d.head_dim, d.rope_base, nullptr);
+            if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; }
+        }
+    }
+    if (st != TASC_OK) {
+        if (m->rope) cudaFree(m->rope);
+        delete m;
+        return st;
+    }
+    *out = m;
+    return TASC_OK;
+}
+
+extern "C" tasc_status tasc_model_destroy(tasc_model* m) {
+    if (!m) return TASC_EINVAL;
+    if (m->rope) cudaFree(m->rope);
+    delete m;
+    return TASC_OK;
+}
+
+extern "C" size_t tasc_workspace_bytes(const tasc_model* m, int32_t B_max, int32_t k_max) {
+    if (!m || B_max < 1 || k_max < 1 || k_max > TASC_MAX_ROWS - 1) return 0;
+    return layout_workspace(m, B_max, nullptr).bytes;
+}
+
+extern "C" tasc_status tasc_prefill(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, int32_t B, int32_t max_len,
+                                    void* workspace, size_t workspace_bytes, tasc_stream stream) {
+    if (!check_common(m, kv, seqs, B, workspace, workspace_bytes) || max_len < 1 || max_len > seqs->stride) return TASC_EINVAL;
+    const Workspace w = layout_workspace(m, B, workspace);
+    return prefill_enqueue(m, kv, seqs, w, B, max_len, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" tasc_status tasc_verify_step(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, const int32_t* drafts,
+                                        int32_t B, int32_t k, const int32_t* forced_targets, int32_t* n_accepted,
+                                        int32_t* next_token, int32_t* target_tokens, float* logits_dbg, void* workspace,
+                                        size_t workspace_bytes, tasc_stream stream) {
+    if (!check_common(m, kv, seqs, B, workspace, workspace_bytes) || !drafts || !n_accepted || !next_token || k < 1 ||
+        k > TASC_MAX_ROWS - 1)
+        return TASC_EINVAL;
+    const Workspace w = layout_workspace(m, B, workspace);
+    return verify_enqueue(m, kv, seqs, w, drafts, B, k, forced_targets, n_accepted, next_token, target_tokens, logits_dbg,
+                          static_cast<cudaStream_t>(stream));
+}
+
+extern "C" tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* dr, const tasc_kv* kv, const tasc_seqs* seqs_in,
+                                     int32_t B, int32_t max_new, const tasc_draft_params* p, int32_t* out, tasc_stats* stats,
+                                     void* workspace, size_t workspace_bytes, tasc_stream stream) {
+    if (!check_common(m, kv, seqs_in, B, workspace, workspace_bytes) || !dr || !p || !out || max_new < 1) return TASC_EINVAL;
+    const int k = p->k;
+    if (k < 1 || k > TASC_MAX_ROWS - 1) return TASC_EINVAL;
+    if (p->mode < TASC_MODE_GREEDY || p->mode > TASC_MODE_FORCED_ACCEPT) return TASC_EINVAL;
+    if (p->mode == TASC_MODE_CONTINUATION && (!p->continuation || p->continuation_stride < (int64_t)max_new + k + 1)) return TASC_EINVAL;
+    if (p->mode == TASC_MODE_FORCED_ACCEPT && (p->forced_accept < 0 || p->forced_accept > k)) return TASC_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const Workspace w = layout_workspace(m, B, workspace);
+
+    std::vector<int32_t> plen(B);
+    TASC_CUDA_TRY(cudaMemcpyAsync(plen.data(), seqs_in->len, B * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    TASC_CUDA_TRY(cudaStreamSynchronize(s));
+    int max_len = 0;
+    for (int b = 0; b < B; ++b) {
+        if (plen[b] < 1 || (int64_t)plen[b] + max_new + k > seqs_in->stride) return TASC_EINVAL;
+        max_len = std::max(max_len, plen[b]);
+    }
+    init_generate_kernel<<<(B + 127) / 128, 128, 0, s>>>(seqs_in->len, w.prompt_len, w.stop_len, B, max_new);
+    TASC_CUDA_TRY(cudaMemsetAsync(w.hist, 0, TASC_MAX_ROWS * sizeof(long long), s));
+    tasc_seqs seqs = *seqs_in;
+    seqs.stop_len = w.stop_len;
+
+    cudaEvent_t ev[3];
+    for (auto& e : ev) TASC_CUDA_TRY(cudaEventCreate(&e));
+    tasc_status st = TASC_OK;
+    cudaEventRecord(ev[0], s);
+    st = prefill_enqueue(m, kv, &seqs, w, B, max_len, s);
+    cudaEventRecord(ev[1], s);
+    int64_t steps = 0;
+    int min_gen = 0;
+    const bool forced = p->mode != TASC_MODE_GREEDY;
+    while (st == TASC_OK && min_gen < max_new) {
+        const int todo = (max_new - min_gen + k) / (k + 1);      // the slowest sequence needs at least this many steps
+        for (int i = 0; i < todo && st == TASC_OK; ++i) {
+            st = tasc_draft(dr, seqs.tokens, seqs.stride, seqs.len, B, k, p->lambda_num, p->lambda_den, w.drafts, s);
+            if (st != TASC_OK) break;
+            if (forced)
+                launch_forced_targets(p->mode, w.drafts, p->continuation, p->continuation_stride, seqs.len, w.prompt_len,
+                                      p->forced_accept, m->desc.vocab, B, k, w.targets, s);
+            st = verify_enqueue(m, kv, &seqs, w, w.drafts, B, k, forced ? w.targets : nullptr, w.n_accepted, w.next_token,
+                                nullptr, nullptr, s);
+            ++steps;
+        }
+        if (st != TASC_OK) break;
+        launch_min_generated(seqs.len, w.prompt_len, B, w.min_gen, s);
+        if (cudaMemcpyAsync(&min_gen, w.min_gen, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; break; }
+        int dev_status = 0;
+        if (cudaMemcpy(&dev_status, w.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; break; }
+        if (dev_status != 0) { st = dev_status; break; }
+    }
+    cudaEventRecord(ev[2], s);
+    if (st == TASC_OK) {
+        launch_gather_output(seqs.tokens, seqs.stride, w.prompt_len, B, max_new, out, s);
+        if (cudaStreamSynchronize(s) != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; }
+    } else {
+        cudaStreamSynchronize(s);
+        (void)cudaGetLastError();
+    }
+    if (stats) {
+        long long hist[TASC_MAX_ROWS] = {0};
+        if (st == TASC_OK && cudaMemcpy(hist, w.hist, sizeof(hist), cudaMemcpyDeviceToHost) != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; }
+        stats->steps = steps;
+        stats->committed = 0;
+        for (int a = 0; a < TASC_MAX_ROWS; ++a) { stats->accepted_hist[a] = hist[a]; stats->committed += hist[a] * (a + 1); }
+        stats->prefill_ms = stats->decode_ms = 0.f;
+        if (st == TASC_OK) {
+            cudaEventElapsedTime(&stats->prefill_ms, ev[0], ev[1]);
+            cudaEventElapsedTime(&stats->decode_ms, ev[1], ev[2]);
+        }
+    }
+    for (auto& e : ev) cudaEventDestroy(e);
+    return st;
+}
+
+extern "C" tasc_status tasc_poll_status(void* workspace, tasc_stream stream) {
+    if (!workspace) return TASC_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int v = 0;
+    TASC_CUDA_TRY(cudaStreamSynchronize(s));
+    TASC_CUDA_TRY(cudaMemcpy(&v, workspace, sizeof(int), cudaMemcpyDeviceToHost));
+    if (v != 0) TASC_CUDA_TRY(cudaMemset(workspace, 0, sizeof(int)));
+    return v;
+}
+
+extern "C" size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K) {
+    if (M < 1 || N < 1 || K < 1) return 0;
+    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40);
+    return 256 + gemm_partial_bytes(p, M, N);
+}
+
+extern "C" tasc_status tasc_gemm_bf16(const void* x, const void* wt, float* y, int32_t M, int32_t N, int32_t K, void* workspace,
+                                      size_t workspace_bytes, tasc_stream stream) {
+    if (!x || !wt || !y || !workspace || M < 1 || N < 1 || K < 8 || K % 8) return TASC_EINVAL;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return TASC_EINVAL;
+    const size_t need = tasc_gemm_workspace_bytes(M, N, K);
+    if (workspace_bytes < need) return TASC_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40);
+    tasc_status st = gemm_set_attributes();
+    if (st != TASC_OK) return st;
+    CUtensorMap tmW, tmX;
+    if ((st = encode_tmap_bf16(&tmW, wt, N, K, 128)) != TASC_OK) return st;
+    if ((st = encode_tmap_bf16(&tmX, x, M, K, p.BN)) != TASC_OK) return st;
+    int* status = static_cast<int*>(workspace);
+    float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
+    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, nullptr, nullptr, status, s)) != TASC_OK) return st;
+    launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
+extern "C" const char* tasc_status_string(tasc_status s) {
+    switch (s) {
+        case TASC_OK: return "ok";
+        case TASC_EINVAL: return "invalid argument";
+        case TASC_ENOMEM: return "out of memory";
+        case TASC_ECUDA: return "CUDA call failed";
+        case TASC_ECAPACITY: return "capacity exceeded";
+        case TASC_ENOKV: return "KV position outside the block table";
+        case TASC_ETIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}

@@ -1,0 +1,269 @@
+// bf16 GEMM for the verify forward on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+//
+// The verify step multiplies a handful of token rows (M = B * (k+1)) by large weight matrices, so
+// the operands are swapped: the weight tile supplies the 128 rows of the MMA (UMMA M = 128), the
+// token rows are the MMA's N (16..256).  D^T[128 weight rows][BN tokens] accumulates in TMEM in
+// float32.  The kernel is weight-bandwidth bound: each CTA streams a [128 x k-range] slab of W
+// through a multi-stage TMA -> shared-memory ring; split-K spreads a matrix with few row tiles
+// over all SMs.  Partial sums go to global memory and are added in fixed order by the consumer
+// kernels, so results do not depend on scheduling.
+//
+// Warp roles (192 threads): warps 0-3 epilogue (TMEM lanes 32w..32w+31), warp 4 TMA producer,
+// warp 5 TMEM allocation + MMA issue.  Every wait is bounded; on timeout the CTA records
+// TASC_ETIMEOUT, skips the remaining work, releases TMEM and returns.
+#include "kernels.h"
+
+#include <algorithm>
+#include <mutex>
+
+namespace tasc {
+
+namespace {
+
+constexpr int BM = 128;           // weight rows per tile (UMMA M)
+constexpr int BK = 64;            // k elements per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int GEMM_THREADS = 192;
+constexpr int ARGMAX_SMEM = 4 * 256 * 8;
+
+struct GemmArgs {
+    float* partials;
+    int M, N, K;
+    int num_kb, splits, m_tiles, BN, stages;
+    unsigned long long* argmax;
+    float* logits;
+    int* status;
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const GemmArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+
+    const int BN = a.BN, stages = a.stages;
+    const uint32_t b_stage_bytes = (uint32_t)BN * BK * 2;
+    const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8u * stages;
+    const uint32_t bar_acc = bar_full + 16u * stages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * stages + 1);
+    unsigned long long* s_arg = reinterpret_cast<unsigned long long*>(bars + 2 * stages + 2);   // [4][256]
+
+    int bid = blockIdx.x;
+    const int m_tile = bid % a.m_tiles; bid /= a.m_tiles;
+    const int split = bid % a.splits;
+    const int out_tile = bid / a.splits;
+    const int kb_begin = (int)(((long long)a.num_kb * split) / a.splits);
+    const int kb_end = (int)(((long long)a.num_kb * (split + 1)) / a.splits);
+    const int n_kb = kb_end - kb_begin;
+    const int f0 = out_tile * BM;       // first weight row (output feature) of the tile
+    const int m0 = m_tile * BN;         // first token row of the tile
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t ncols = 32;
+    while ((int)ncols < BN) ncols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(bar_full + 8u * s, 1);
+            mbar_init(bar_empty + 8u * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        fence_barrier_init();
+    }
+    if (warp == 4 && lane == 0) {
+        tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmX);
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(tmem_slot), ncols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first();   // weights are read once per step
+            const uint64_t pol_x = policy_evict_last();    // the token rows are re-read by every CTA
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % stages;
+                const uint32_t round = (uint32_t)(i / stages);
+                if (!mbar_wait(bar_empty + 8u * s, (round & 1u) ^ 1u)) { set_status(a.status, TASC_ETIMEOUT); break; }
+                const uint32_t dstA = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint32_t dstB = dstA + A_STAGE_BYTES;
+                mbar_expect_tx(bar_full + 8u * s, stage_bytes);
+                const int kc = (kb_begin + i) * BK;
+                tma_load_2d_hint(dstA, &tmW, kc, f0, bar_full + 8u * s, pol_w);
+                tma_load_2d_hint(dstB, &tmX, kc, m0, bar_full + 8u * s, pol_x);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+            bool ok = true;
+            for (int i = 0; i < n_kb && ok; ++i) {
+                const int s = i % stages;
+                const uint32_t round = (uint32_t)(i / stages);
+                if (!mbar_wait(bar_full + 8u * s, round & 1u)) { set_status(a.status, TASC_ETIMEOUT); ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                    const uint64_t da = umma_desc_k_sw128(sa + kk * UMMA_K * 2);
+                    const uint64_t db = umma_desc_k_sw128(sb + kk * UMMA_K * 2);
+                    umma_bf16(tmem_base, da, db, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(bar_empty + 8u * s);     // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(bar_acc);            // accumulator complete
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 0..3)
+        bool have = n_kb > 0;
+        if (have) {
+            if (!mbar_wait(bar_acc, 0)) { set_status(a.status, TASC_ETIMEOUT); have = false; }
+        }
+        tc_fence_after();
+        const int f = f0 + warp * 32 + lane;
+        const bool f_ok = f < a.N;
+        for (int c = 0; c < BN / 16; ++c) {
+            uint32_t r[16];
+            if (have) {
+                tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 16), r);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) r[j] = 0u;
+            }
+            if (a.argmax) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int n = c * 16 + j;
+                    const uint32_t key = f_ok ? float_key(__uint_as_float(r[j])) : 0u;
+                    const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
+                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
+                    if (lane == 0) {
+                        const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
+                        s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
+                    }
+                    if (a.logits && f_ok && m0 + n < a.M) a.logits[(size_t)(m0 + n) * a.N + f] = __uint_as_float(r[j]);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int m = m0 + c * 16 + j;
+                    if (f_ok && m < a.M) a.partials[((size_t)split * a.M + m) * a.N + f] = __uint_as_float(r[j]);
+                }
+            }
+        }
+        if (a.argmax) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int n = threadIdx.x; n < BN; n += 128) {
+                if (m0 + n < a.M) {
+                    unsigned long long best = s_arg[n];
+                    best = max(best, s_arg[256 + n]);
+                    best = max(best, s_arg[512 + n]);
+                    best = max(best, s_arg[768 + n]);
+                    atomicMax(&a.argmax[m0 + n], best);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem_base, ncols);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    });
+    return fn;
+}
+
+int stage_bytes_for(int BN) { return A_STAGE_BYTES + BN * BK * 2; }
+int smem_for(int BN, int stages) { return 1024 + stages * stage_bytes_for(BN) + (2 * stages + 2) * 8 + ARGMAX_SMEM; }
+
+}  // namespace
+
+tasc_status encode_tmap_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return TASC_ECUDA;
+    if ((reinterpret_cast<uintptr_t>(ptr) & 15u) || (cols % 8u) || box_rows == 0 || box_rows > 256) return TASC_EINVAL;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TASC_OK : TASC_ECUDA;
+}
+
+GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes) {
+    GemmPlan p;
+    p.m_tiles = (M + 255) / 256;
+    int per = (M + p.m_tiles - 1) / p.m_tiles;
+    p.BN = std::max(16, (per + 15) / 16 * 16);
+    p.m_tiles = (M + p.BN - 1) / p.BN;
+    p.out_tiles = (N + BM - 1) / BM;
+    const int num_kb = (K + BK - 1) / BK;
+    const int tiles = p.out_tiles * p.m_tiles;
+    // Enough CTAs to cover the 148 SMs about twice, each keeping at least two k-blocks.
+    int s = std::max(1, (296 + tiles / 2) / tiles);
+    s = std::min(s, std::max(1, num_kb / 2));
+    while (s > 1 && (size_t)s * M * N * sizeof(float) > max_partial_bytes) --s;
+    p.splits = s;
+    const int kb_per = (num_kb + s - 1) / s;
+    // Two CTAs per SM when the tile is small (about 110 KB each), otherwise one deep ring.
+    const int budget = p.BN <= 64 ? 100 * 1024 : 190 * 1024;
+    int st = budget / stage_bytes_for(p.BN);
+    st = std::max(2, std::min(st, 8));
+    st = std::min(st, std::max(2, kb_per));
+    p.stages = st;
+    p.smem_bytes = smem_for(p.BN, st);
+    return p;
+}
+
+tasc_status gemm_set_attributes() {
+    TASC_CUDA_TRY(cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    return TASC_OK;
+}
+
+tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, float* partials, int M, int N, int K,
+                             const GemmPlan& plan, unsigned long long* argmax, float* logits, int* status,
+                             cudaStream_t stream) {
+    if (M <= 0 || N <= 0 || K <= 0) return TASC_EINVAL;
+    if (argmax && plan.splits != 1) return TASC_EINVAL;
+    GemmArgs a;
+    a.partials = partials; a.M = M; a.N = N; a.K = K;
+    a.num_kb = (K + BK - 1) / BK; a.splits = plan.splits; a.m_tiles = plan.m_tiles; a.BN = plan.BN; a.stages = plan.stages;
+    a.argmax = argmax; a.logits = logits; a.status = status;
+    const int grid = plan.out_tiles * plan.splits * plan.m_tiles;
+    gemm_bf16_kernel<<<grid, GEMM_THREADS, plan.smem_bytes, stream>>>(*tmW, *tmX, a);
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
+}  // namespace tasc

@@ -1,0 +1,94 @@
+// Internal launch interface between the C-ABI layer (api.cu) and the kernel files.
+#pragma once
+
+#include "common.cuh"
+
+namespace tasc {
+
+// ------------------------------------------------------------------ tensor-core GEMM (gemm_tcgen05.cu)
+// Computes partial sums P[s][m][n] = sum over the k-range of split s of X[m][k] * W[n][k]
+// (bf16 inputs, float32 accumulation in TMEM).  Consumers add the `splits` slices in order.
+struct GemmPlan {
+    int BN;          // token rows per CTA tile (UMMA N), multiple of 16, 16..256
+    int m_tiles;     // ceil(M / BN)
+    int out_tiles;   // ceil(N / 128): weight rows per CTA tile = UMMA M = 128
+    int splits;      // split-K factor
+    int stages;      // TMA -> MMA pipeline depth
+    int smem_bytes;
+};
+GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes);
+inline size_t gemm_partial_bytes(const GemmPlan& p, int M, int N) { return (size_t)p.splits * M * N * sizeof(float); }
+
+// rows x cols bf16 row-major matrix, box = {64 cols, box_rows}, 128-byte swizzle.
+tasc_status encode_tmap_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+// argmax != null: LM-head mode (splits must be 1): per token row an atomic max of (value, id) is kept in
+// argmax[m] instead of writing partials; `logits` (nullable) additionally receives the full rows.
+tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, float* partials, int M, int N, int K,
+                             const GemmPlan& plan, unsigned long long* argmax, float* logits, int* status,
+                             cudaStream_t stream);
+tasc_status gemm_set_attributes();
+
+// ------------------------------------------------------------------ float32 GEMM for the f32 model (gemm_simt.cu)
+// Same contract with splits = 1: P[0][m][n].
+void launch_gemm_f32(const float* X, const float* W, float* partials, int M, int N, int K,
+                     unsigned long long* argmax, float* logits, cudaStream_t stream);
+
+// ------------------------------------------------------------------ layer kernels (layers.cu)
+struct RowPlan {              // per-step row bookkeeping, all device pointers into the workspace
+    int* row_tok;             // [M] token id of each row
+    int* row_pos;             // [M] position of each row, -1 = row not in use
+    int* seq_pos0;            // [B] position of the sequence's first row
+    int* seq_rows;            // [B] rows in use (0 = sequence skipped)
+};
+// Rows of a verify step: [last committed token, drafts] at positions len-1 ..; skipped when len >= stop_len.
+void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len,
+                        const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
+                        cudaStream_t stream);
+// Rows of prefill chunk c: committed tokens c*R .. c*R+R-1, limited to positions <= len-2.
+void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
+                         int chunk, int vocab, int* status, cudaStream_t stream);
+
+template <typename T>
+void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
+                       cudaStream_t stream);
+// x += sum_s P[s]; h = RMSNorm(x) * gain  (gain == null: only the residual update)
+template <typename T>
+void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,
+                          cudaStream_t stream);
+// qkv = sum_s P[s]; RoPE on q and k; q -> qbuf [M][n_q*hd]; k, v -> KV pages of the layer.
+template <typename T>
+void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp, const float2* rope, T* qbuf,
+                            T* k_pages, T* v_pages, const int32_t* block_table, int max_pages, int page_size,
+                            long long n_pages, int M, int R, int n_q, int n_kv, int hd, int max_positions, int* status,
+                            cudaStream_t stream);
+// act = SiLU(gate) * up with gate = sum_s P[s][:, :dff], up = sum_s P[s][:, dff:]
+template <typename T>
+void launch_silu_mul(const float* partials, int splits, T* act, int M, int dff, cudaStream_t stream);
+// y[M][N] = sum_s P[s]
+void launch_sum_partials(const float* partials, int splits, float* y, size_t n, cudaStream_t stream);
+void launch_fill_u64(unsigned long long* p, unsigned long long v, int n, cudaStream_t stream);
+// Greedy acceptance, commit and bookkeeping (one thread per sequence).
+void launch_accept(const unsigned long long* argmax, const RowPlan& rp, const int32_t* drafts,
+                   const int32_t* forced_targets, int32_t* tokens, int64_t stride, int32_t* len, int B, int R,
+                   int32_t* n_accepted, int32_t* next_token, int32_t* target_tokens, long long* hist,
+                   cudaStream_t stream);
+void launch_rope_table(float2* table, int max_positions, int hd, float base, cudaStream_t stream);
+// Teacher-forced targets built on the device from the drafts (see TASC_MODE_*).
+void launch_forced_targets(int mode, const int32_t* drafts, const int32_t* continuation, int64_t cont_stride,
+                           const int32_t* len, const int32_t* prompt_len, int forced_accept, int vocab, int B, int k,
+                           int32_t* targets, cudaStream_t stream);
+void launch_gather_output(const int32_t* tokens, int64_t stride, const int32_t* prompt_len, int B, int max_new,
+                          int32_t* out, cudaStream_t stream);
+void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, int* out_min, cudaStream_t stream);
+
+// ------------------------------------------------------------------ attention (attention.cu)
+// Verify attention of R query rows per sequence over the paged KV cache (grouped-query, causal within the rows).
+template <typename T>
+void launch_attention(const T* qbuf, const T* k_pages, const T* v_pages, const int32_t* block_table, int max_pages,
+                      int page_size, long long n_pages, const RowPlan& rp, T* out, float* scratch, int B, int R, int n_q,
+                      int n_kv, int hd, int n_splits, cudaStream_t stream);
+size_t attention_scratch_bytes(int B, int R, int n_q, int hd, int n_splits);
+int attention_splits(int B, int n_kv, int max_ctx);
+
+}  // namespace tasc

@@ -1,0 +1,121 @@
+"""Verify step and generation loop against the oracle, replayed in lock-step (the oracle's committed
+state is fed to the device at every step, so one near-tie cannot derail the rest of the comparison)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decode as G
+from tests.gpu_harness import lockstep, make_setup, need_gpu
+from workload import configs, corpus
+
+# logits tolerance: float32 model 1e-4 absolute; bf16 models max-abs 2e-2 / relative 1e-2.
+# token rule: a device argmax may differ from the oracle's only where the oracle's top-2 gap is below gap_tol.
+F32_TOL = dict(logit_atol=1e-4, logit_rtol=0.0, gap_tol=2e-4)
+BF16_TOL = dict(logit_atol=2e-2, logit_rtol=1e-2, gap_tol=1e-2)
+
+
+def check(rep, max_near_tie_frac=0.25):
+    assert rep.steps > 0
+    assert rep.draft_mismatches == 0, "drafts must be bit-exact"
+    assert not rep.hard_mismatches, rep.hard_mismatches[:5]
+    assert rep.accept_mismatches == 0
+    assert rep.near_tie_mismatches <= max_near_tie_frac * rep.rows
+    print(f"lockstep: steps={rep.steps} rows={rep.rows} near_tie_mismatches={rep.near_tie_mismatches} "
+          f"max_logit_err={rep.max_logit_err:.3e}")
+
+
+@pytest.mark.gpu
+def test_config0_lockstep_full():
+    cfg = configs.get(0)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 1)
+    check(lockstep(s, prompts, cfg.max_new, cfg.k, **F32_TOL))
+
+
+@pytest.mark.gpu
+def test_config0_batch_with_gain_jitter_and_ragged_prompts():
+    cfg = configs.get(0)
+    s = make_setup(cfg, gain_jitter=0.2)
+    prompts = corpus.make_prompts(cfg, 5, prompt_len=37)          # 37: prefill ends in a ragged chunk
+    check(lockstep(s, prompts, 24, 7, **F32_TOL))
+
+
+@pytest.mark.gpu
+def test_config0_teacher_forced_accept_lengths():
+    cfg = configs.get(0)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 3)
+    for a in (0, 2, cfg.k):
+        rep = lockstep(s, prompts, 20, cfg.k, oracle_kwargs=[dict(forced_accept=a)] * 3, forced_mode="accept", **F32_TOL)
+        check(rep)
+
+
+@pytest.mark.gpu
+def test_config0_generate_matches_oracle_and_plain_greedy():
+    b = need_gpu()
+    cfg = configs.get(0)
+    s = make_setup(cfg)
+    B = 4
+    prompts = corpus.make_prompts(cfg, B)
+    P = prompts.shape[1]
+    stride = P + cfg.max_new + cfg.k + 1
+    tokens = torch.zeros((B, stride), dtype=torch.int32, device="cuda")
+    tokens[:, :P] = torch.from_numpy(prompts).cuda()
+    length = torch.full((B,), P, dtype=torch.int32, device="cuda")
+    pool, bt, kv = s.model.new_kv(B, stride + b.MAX_ROWS)
+    ws = s.model.new_workspace(B, cfg.k)
+    out, st = b.tasc_generate(s.model, s.drafter, kv, b.make_seqs(tokens, length), B, cfg.max_new, cfg.k, ws)
+    out = out.cpu().numpy()
+    assert st.steps >= cfg.max_new // (cfg.k + 1) and st.committed >= B * cfg.max_new
+    assert sum(st.accepted_hist) > 0 and st.decode_ms > 0
+    for i in range(B):
+        spec = G.greedy_speculative(s.oracle, s.ngrams, prompts[i], cfg.max_new, cfg.k)
+        gaps = [g for stp in spec.steps for g in stp.gap]
+        want = np.array(spec.tokens)
+        if not np.array_equal(out[i], want):
+            first = int(np.argmax(out[i] != want))
+            assert min(gaps) < F32_TOL["gap_tol"], f"sequence {i} diverges at {first} without a near-tie"
+    # the committed tokens on the device equal the returned output
+    tok = tokens.cpu().numpy()
+    assert np.array_equal(tok[:, P:P + cfg.max_new], out)
+    assert (length.cpu().numpy() >= P + cfg.max_new).all()
+
+
+@pytest.mark.gpu
+def test_kv_exhaustion_is_reported_not_faulted():
+    b = need_gpu()
+    cfg = configs.get(0)
+    s = make_setup(cfg, build_drafter=False, oracle_ngrams=False)
+    B, P, k = 1, 32, 4
+    tokens = torch.zeros((B, 64), dtype=torch.int32, device="cuda")
+    tokens[:, :P] = torch.from_numpy(corpus.make_prompts(cfg, B)).cuda()
+    length = torch.full((B,), P, dtype=torch.int32, device="cuda")
+    pool, bt, kv = s.model.new_kv(B, 32)           # two pages: positions 0..31 only
+    ws = s.model.new_workspace(B, k)
+    seqs = b.make_seqs(tokens, length)
+    b.tasc_prefill(s.model, kv, seqs, B, P, ws)
+    b.tasc_poll_status(ws)
+    drafts = torch.zeros((B, k), dtype=torch.int32, device="cuda")
+    b.tasc_verify_step(s.model, kv, seqs, drafts, ws)       # rows at positions 31..35: 32.. have no page
+    with pytest.raises(b.TascError) as e:
+        b.tasc_poll_status(ws)
+    assert e.value.code == b.ENOKV
+    b.tasc_poll_status(ws)                                  # cleared
+
+
+@pytest.mark.gpu
+def test_verify_rejects_bad_arguments():
+    b = need_gpu()
+    cfg = configs.get(0)
+    s = make_setup(cfg, build_drafter=False, oracle_ngrams=False)
+    tokens = torch.zeros((1, 64), dtype=torch.int32, device="cuda")
+    length = torch.ones(1, dtype=torch.int32, device="cuda")
+    pool, bt, kv = s.model.new_kv(1, 64)
+    seqs = b.make_seqs(tokens, length)
+    small = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(b.TascError) as e:
+        b.tasc_verify_step(s.model, kv, seqs, torch.zeros((1, 4), dtype=torch.int32, device="cuda"), small)
+    assert e.value.code == b.EINVAL
+    ws = s.model.new_workspace(1, 4)
+    with pytest.raises(b.TascError):
+        b.tasc_verify_step(s.model, kv, seqs, torch.zeros((1, 16), dtype=torch.int32, device="cuda"), ws)   # k + 1 > 16
