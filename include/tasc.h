@@ -242,6 +242,14 @@ tasc_status tasc_poll_status(void* workspace, tasc_stream stream);
  */
 tasc_status tasc_gemm_bf16(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                            void* workspace, size_t workspace_bytes, tasc_stream stream);
+/*
+ * Same product for float32 X: every x is carried through the bf16 tensor cores as the pair
+ * hi = bf16(x), lo = bf16(x - hi), and the two partial products are added in float32.  This is how
+ * the verify forward feeds its activations to the projections, so that only the weights and the
+ * KV cache are rounded to bf16.   x: device, float32[M][K].  Other arguments as tasc_gemm_bf16.
+ */
+tasc_status tasc_gemm_bf16x2(const float* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                             void* workspace, size_t workspace_bytes, tasc_stream stream);
 size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
 
 const char* tasc_status_string(tasc_status s);

@@ -86,6 +86,8 @@ lib.tasc_generate.argtypes = [_P, _P, C.POINTER(Kv), C.POINTER(Seqs), C.c_int32,
                               C.POINTER(Stats), _P, C.c_size_t, _P]
 lib.tasc_poll_status.argtypes = [_P, _P]
 lib.tasc_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
+lib.tasc_gemm_bf16x2.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
+lib.tasc_gemm_bf16x2.restype = C.c_int32
 lib.tasc_gemm_workspace_bytes.restype = C.c_size_t
 lib.tasc_gemm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
 for _f in ("tasc_drafter_build", "tasc_drafter_export", "tasc_drafter_destroy", "tasc_draft", "tasc_model_create",
@@ -273,6 +275,19 @@ def tasc_gemm_bf16(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
     ws = torch.zeros(max(nbytes, 256), dtype=torch.uint8, device=x.device)
     y = torch.empty((M, N), dtype=torch.float32, device=x.device)
     _check(lib.tasc_gemm_bf16(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(ws), ws.numel(), _stream()), "tasc_gemm_bf16")
+    tasc_poll_status(ws)
+    return y
+
+
+def tasc_gemm_bf16x2(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
+    """Y[M, N] float32 = X[M, K] @ W[N, K]^T for float32 X (carried as hi/lo bf16 pairs) and bf16 W."""
+    _dev(x, torch.float32)
+    _dev(w, torch.bfloat16)
+    M, K = x.shape
+    N = w.shape[0]
+    ws = torch.zeros(max(lib.tasc_gemm_workspace_bytes(M, N, K), 256), dtype=torch.uint8, device=x.device)
+    y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    _check(lib.tasc_gemm_bf16x2(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(ws), ws.numel(), _stream()), "tasc_gemm_bf16x2")
     tasc_poll_status(ws)
     return y
 

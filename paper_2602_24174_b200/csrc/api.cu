@@ -44,7 +44,8 @@ struct Workspace {
     unsigned long long* argmax;   // [M]
     int32_t *drafts, *targets, *n_accepted, *next_token, *prompt_len, *stop_len;
     float* x;                     // [M][d] residual stream
-    void *h, *q, *o, *act;        // model dtype
+    void *h, *o, *act;            // GEMM inputs: float rows, or (hi, lo) bf16 row pairs
+    float* q;                     // [M][n_q * hd]
     float* partials;
     size_t partial_bytes;
     float* att_scratch;
@@ -74,10 +75,12 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     w.prompt_len = L.take<int32_t>(base, B);
     w.stop_len = L.take<int32_t>(base, B);
     w.x = L.take<float>(base, M * d.d_model);
-    w.h = L.take<uint8_t>(base, M * d.d_model * esz);
-    w.q = L.take<uint8_t>(base, M * m->q_dim * esz);
-    w.o = L.take<uint8_t>(base, M * m->q_dim * esz);
-    w.act = L.take<uint8_t>(base, M * d.d_ff * esz);
+    // bf16: two rows per token plus tile padding (tiles of at most 128 tokens, rounded up to 16)
+    const size_t act_rows = d.dtype == TASC_F32 ? M : 2 * (M + 16 * (M / 128 + 1));
+    w.h = L.take<uint8_t>(base, act_rows * d.d_model * esz);
+    w.q = L.take<float>(base, M * m->q_dim);
+    w.o = L.take<uint8_t>(base, act_rows * m->q_dim * esz);
+    w.act = L.take<uint8_t>(base, act_rows * d.d_ff * esz);
     const size_t n_max = std::max<size_t>({(size_t)m->qkv_rows, (size_t)2 * d.d_ff, (size_t)d.d_model});
     w.partial_bytes = std::max(MIN_PARTIAL_BYTES, M * n_max * sizeof(float));
     w.partials = L.take<float>(base, w.partial_bytes / sizeof(float));
@@ -117,7 +120,7 @@ tasc_status run_gemm(const tasc_model* m, const Workspace& w, const void* X, con
         return TASC_OK;
     } else {
         (void)X; (void)W;
-        GemmPlan plan = plan_gemm(M, N, K, w.partial_bytes);
+        GemmPlan plan = plan_gemm(M, N, K, w.partial_bytes, true);
         if (argmax) plan.splits = 1;
         *splits = plan.splits;
         return launch_gemm_bf16(tmW, tmX, w.partials, M, N, K, plan, argmax, logits, w.status, s);
@@ -133,18 +136,20 @@ tasc_status forward(const tasc_model* m, const tasc_kv* kv, const Workspace& w, 
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
     const int att_splits = attention_splits(B, d.n_kv_heads, max_ctx);
     CUtensorMap tm_h, tm_o, tm_act;
+    int TB = 0;
     if constexpr (sizeof(T) == 2) {
-        const GemmPlan p = plan_gemm(M, d.d_model, d.d_model, w.partial_bytes);      // BN depends on M only
+        TB = gemm_token_tile(M, true);                      // token tile depends on M only
+        const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
         tasc_status st;
-        if ((st = encode_tmap_bf16(&tm_h, w.h, M, d.d_model, p.BN)) != TASC_OK) return st;
-        if ((st = encode_tmap_bf16(&tm_o, w.o, M, m->q_dim, p.BN)) != TASC_OK) return st;
-        if ((st = encode_tmap_bf16(&tm_act, w.act, M, d.d_ff, p.BN)) != TASC_OK) return st;
+        if ((st = encode_tmap_bf16(&tm_h, w.h, rows, d.d_model, 2 * TB)) != TASC_OK) return st;
+        if ((st = encode_tmap_bf16(&tm_o, w.o, rows, m->q_dim, 2 * TB)) != TASC_OK) return st;
+        if ((st = encode_tmap_bf16(&tm_act, w.act, rows, d.d_ff, 2 * TB)) != TASC_OK) return st;
     }
     T* h = static_cast<T*>(w.h);
-    T* q = static_cast<T*>(w.q);
+    float* q = w.q;
     T* o = static_cast<T*>(w.o);
     T* act = static_cast<T*>(w.act);
-    launch_embed_norm<T>(static_cast<const T*>(m->embed), w.rp.row_tok, m->attn_norm[0], d.rms_eps, w.x, h, M, d.d_model, s);
+    launch_embed_norm<T>(static_cast<const T*>(m->embed), w.rp.row_tok, m->attn_norm[0], d.rms_eps, w.x, h, M, d.d_model, TB, s);
     for (int l = 0; l < d.n_layers; ++l) {
         const KvView kvl = layer_kv(m, kv, l);
         int sp = 1;
@@ -156,18 +161,18 @@ tasc_status forward(const tasc_model* m, const tasc_kv* kv, const Workspace& w, 
                                   kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, M, R, d.n_q_heads,
                                   d.n_kv_heads, d.head_dim, d.max_positions, w.status, s);
         launch_attention<T>(q, static_cast<const T*>(kvl.k), static_cast<const T*>(kvl.v), kv->block_table,
-                            kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, w.att_scratch, B, R, d.n_q_heads,
+                            kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, w.att_scratch, B, R, d.n_q_heads,
                             d.n_kv_heads, d.head_dim, att_splits, s);
         st = run_gemm<T>(m, w, o, &tm_o, m->wo[l], bf ? &m->tm_o[l] : nullptr, M, d.d_model, m->q_dim, &sp, nullptr, nullptr, s);
         if (st != TASC_OK) return st;
-        launch_residual_norm<T>(w.partials, sp, w.x, m->mlp_norm[l], d.rms_eps, h, M, d.d_model, s);
+        launch_residual_norm<T>(w.partials, sp, w.x, m->mlp_norm[l], d.rms_eps, h, M, d.d_model, TB, s);
         st = run_gemm<T>(m, w, h, &tm_h, m->w_gate_up[l], bf ? &m->tm_gu[l] : nullptr, M, 2 * d.d_ff, d.d_model, &sp, nullptr, nullptr, s);
         if (st != TASC_OK) return st;
-        launch_silu_mul<T>(w.partials, sp, act, M, d.d_ff, s);
+        launch_silu_mul<T>(w.partials, sp, act, M, d.d_ff, TB, s);
         st = run_gemm<T>(m, w, act, &tm_act, m->w_down[l], bf ? &m->tm_down[l] : nullptr, M, d.d_model, d.d_ff, &sp, nullptr, nullptr, s);
         if (st != TASC_OK) return st;
         const float* next_gain = l + 1 < d.n_layers ? m->attn_norm[l + 1] : m->final_norm;
-        launch_residual_norm<T>(w.partials, sp, w.x, next_gain, d.rms_eps, h, M, d.d_model, s);
+        launch_residual_norm<T>(w.partials, sp, w.x, next_gain, d.rms_eps, h, M, d.d_model, TB, s);
     }
     if (lm_head) {
         int sp = 1;
@@ -406,8 +411,10 @@ extern "C" tasc_status tasc_poll_status(void* workspace, tasc_stream stream) {
 
 extern "C" size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K) {
     if (M < 1 || N < 1 || K < 1) return 0;
-    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40);
-    return 256 + gemm_partial_bytes(p, M, N);
+    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40, false);
+    const GemmPlan p2 = plan_gemm(M, N, K, (size_t)1 << 40, true);
+    const size_t split_rows = (size_t)p2.m_tiles * p2.BN * K * 2;      // (hi, lo) copy of X for tasc_gemm_bf16x2
+    return 256 + std::max(gemm_partial_bytes(p, M, N), gemm_partial_bytes(p2, M, N)) + 256 + split_rows;
 }
 
 extern "C" tasc_status tasc_gemm_bf16(const void* x, const void* wt, float* y, int32_t M, int32_t N, int32_t K, void* workspace,
@@ -417,7 +424,7 @@ extern "C" tasc_status tasc_gemm_bf16(const void* x, const void* wt, float* y, i
     const size_t need = tasc_gemm_workspace_bytes(M, N, K);
     if (workspace_bytes < need) return TASC_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40);
+    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40, false);
     tasc_status st = gemm_set_attributes();
     if (st != TASC_OK) return st;
     CUtensorMap tmW, tmX;
@@ -425,6 +432,32 @@ extern "C" tasc_status tasc_gemm_bf16(const void* x, const void* wt, float* y, i
     if ((st = encode_tmap_bf16(&tmX, x, M, K, p.BN)) != TASC_OK) return st;
     int* status = static_cast<int*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
+    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, nullptr, nullptr, status, s)) != TASC_OK) return st;
+    launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
+extern "C" tasc_status tasc_gemm_bf16x2(const float* x, const void* wt, float* y, int32_t M, int32_t N, int32_t K,
+                                        void* workspace, size_t workspace_bytes, tasc_stream stream) {
+    if (!x || !wt || !y || !workspace || M < 1 || N < 1 || K < 8 || K % 8) return TASC_EINVAL;
+    if (reinterpret_cast<uintptr_t>(workspace) % 256) return TASC_EINVAL;
+    if (workspace_bytes < tasc_gemm_workspace_bytes(M, N, K)) return TASC_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40, true);
+    tasc_status st = gemm_set_attributes();
+    if (st != TASC_OK) return st;
+    int* status = static_cast<int*>(workspace);
+    uint8_t* base = static_cast<uint8_t*>(workspace) + 256;
+    float* partials = reinterpret_cast<float*>(base);
+    const size_t pb = (gemm_partial_bytes(p, M, N) + 255) / 256 * 256;
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(base + pb);
+    const uint64_t rows = (uint64_t)p.m_tiles * p.BN;
+    TASC_CUDA_TRY(cudaMemsetAsync(xs, 0, rows * K * 2, s));
+    launch_split_rows(x, xs, M, K, p.TB, s);
+    CUtensorMap tmW, tmX;
+    if ((st = encode_tmap_bf16(&tmW, wt, N, K, 128)) != TASC_OK) return st;
+    if ((st = encode_tmap_bf16(&tmX, xs, rows, K, p.BN)) != TASC_OK) return st;
     if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, nullptr, nullptr, status, s)) != TASC_OK) return st;
     launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
     TASC_CUDA_TRY(cudaGetLastError());

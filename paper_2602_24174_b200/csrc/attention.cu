@@ -72,13 +72,13 @@ attention_split_kernel(const AttArgs a) {
     const int k_begin = sp * chunk;
     const int k_end = min(total, k_begin + chunk);
 
-    const T* q = static_cast<const T*>(a.q);
+    const float* q = static_cast<const float*>(a.q);
     const int qd = a.n_q * hd;
     for (int i = threadIdx.x; i < G * hd; i += ATT_THREADS) {
         const int r = i / hd, d = i % hd;
         const int hl = r / a.R, rr = r % a.R;
         float v = 0.f;
-        if (rr < rows) v = Num<T>::to_f(q[(size_t)(b * a.R + rr) * qd + (kh * g + hl) * hd + d]) * a.scale;
+        if (rr < rows) v = q[(size_t)(b * a.R + rr) * qd + (kh * g + hl) * hd + d] * a.scale;
         Qs[i] = v;
         Os[i] = 0.f;
     }
@@ -151,12 +151,12 @@ attention_split_kernel(const AttArgs a) {
 template <typename T>
 __global__ void __launch_bounds__(128)
 attention_combine_kernel(const float* __restrict__ o_part, const float2* __restrict__ ml_part, RowPlan rp, T* __restrict__ out,
-                         int R, int n_q, int hd, int splits) {
+                         int TB, int R, int n_q, int hd, int splits) {
     const int rr = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const size_t slot0 = (((size_t)b * n_q + h) * R + rr) * splits;
-    T* dst = out + (size_t)(b * R + rr) * n_q * hd + (size_t)h * hd;
+    const int m = b * R + rr, ld = n_q * hd;
     if (rr >= rp.seq_rows[b]) {
-        for (int d = threadIdx.x; d < hd; d += blockDim.x) dst[d] = Num<T>::from_f(0.f);
+        for (int d = threadIdx.x; d < hd; d += blockDim.x) ActStore<T>::put(out, m, h * hd + d, ld, TB, 0.f);
         return;
     }
     float mx = -INFINITY;
@@ -172,7 +172,7 @@ attention_combine_kernel(const float* __restrict__ o_part, const float2* __restr
             const float m = ml_part[slot0 + s].x;
             if (m != -INFINITY) acc += expf(m - mx) * o_part[(slot0 + s) * hd + d];
         }
-        dst[d] = Num<T>::from_f(acc / den);
+        ActStore<T>::put(out, m, h * hd + d, ld, TB, acc / den);
     }
 }
 
@@ -196,9 +196,9 @@ size_t attention_scratch_bytes(int B, int R, int n_q, int hd, int n_splits) {
 }
 
 template <typename T>
-void launch_attention(const T* qbuf, const T* k_pages, const T* v_pages, const int32_t* block_table, int max_pages,
-                      int page_size, long long n_pages, const RowPlan& rp, T* out, float* scratch, int B, int R, int n_q,
-                      int n_kv, int hd, int n_splits, cudaStream_t stream) {
+void launch_attention(const float* qbuf, const T* k_pages, const T* v_pages, const int32_t* block_table, int max_pages,
+                      int page_size, long long n_pages, const RowPlan& rp, T* out, int TB, float* scratch, int B, int R,
+                      int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream) {
     AttArgs a;
     a.q = qbuf; a.kp = k_pages; a.vp = v_pages; a.block_table = block_table;
     a.max_pages = max_pages; a.page_size = page_size; a.n_pages = n_pages; a.rp = rp;
@@ -216,13 +216,13 @@ void launch_attention(const T* qbuf, const T* k_pages, const T* v_pages, const i
         done = true;
     }
     attention_split_kernel<T><<<dim3(n_splits, n_kv, B), ATT_THREADS, smem, stream>>>(a);
-    attention_combine_kernel<T><<<dim3(R, n_q, B), hd < 128 ? 64 : 128, 0, stream>>>(a.o_part, a.ml_part, rp, out, R, n_q, hd, n_splits);
+    attention_combine_kernel<T><<<dim3(R, n_q, B), hd < 128 ? 64 : 128, 0, stream>>>(a.o_part, a.ml_part, rp, out, TB, R, n_q, hd, n_splits);
 }
 
 template void launch_attention<float>(const float*, const float*, const float*, const int32_t*, int, int, long long,
-                                      const RowPlan&, float*, float*, int, int, int, int, int, int, cudaStream_t);
-template void launch_attention<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
-                                              const int32_t*, int, int, long long, const RowPlan&, __nv_bfloat16*, float*,
-                                              int, int, int, int, int, int, cudaStream_t);
+                                      const RowPlan&, float*, int, float*, int, int, int, int, int, int, cudaStream_t);
+template void launch_attention<__nv_bfloat16>(const float*, const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*, int,
+                                              int, long long, const RowPlan&, __nv_bfloat16*, int, float*, int, int, int, int,
+                                              int, int, cudaStream_t);
 
 }  // namespace tasc

@@ -34,6 +34,25 @@ template <> struct Num<__nv_bfloat16> {
     static __device__ __forceinline__ __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
 };
 
+// Activation buffers that feed the GEMMs.  float32 model: plain rows [M][ld].  bf16 model: each value is
+// stored as hi = bf16(v) and lo = bf16(v - hi) in two rows of a tile-local layout: tile t of TB tokens
+// occupies rows [t * 2 TB, t * 2 TB + TB) (hi) and the next TB rows (lo).
+template <typename T> struct ActStore;
+template <> struct ActStore<float> {
+    static __device__ __forceinline__ void put(float* buf, int m, int j, int ld, int TB, float v) {
+        (void)TB;
+        buf[(size_t)m * ld + j] = v;
+    }
+};
+template <> struct ActStore<__nv_bfloat16> {
+    static __device__ __forceinline__ void put(__nv_bfloat16* buf, int m, int j, int ld, int TB, float v) {
+        const size_t row = (size_t)(m / TB) * (2 * TB) + (m % TB);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        buf[row * ld + j] = hi;
+        buf[(row + TB) * ld + j] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+};
+
 // Order-preserving map float -> uint32 (larger float <-> larger key).
 __device__ __forceinline__ uint32_t float_key(float v) {
     uint32_t b = __float_as_uint(v);

@@ -8,6 +8,11 @@
 // over all SMs.  Partial sums go to global memory and are added in fixed order by the consumer
 // kernels, so results do not depend on scheduling.
 //
+// Paired mode (the forward's activations): a float32 activation v is carried as two bf16 rows,
+// hi = bf16(v) and lo = bf16(v - hi), stored tile by tile as [TB hi rows][TB lo rows] (BN = 2 TB).
+// Both halves go through the same MMA and the epilogue adds accumulator columns j and j + TB, so
+// the product keeps about 16 mantissa bits of the activation at no extra weight traffic.
+//
 // Warp roles (192 threads): warps 0-3 epilogue (TMEM lanes 32w..32w+31), warp 4 TMA producer,
 // warp 5 TMEM allocation + MMA issue.  Every wait is bounded; on timeout the CTA records
 // TASC_ETIMEOUT, skips the remaining work, releases TMEM and returns.
@@ -31,6 +36,7 @@ struct GemmArgs {
     float* partials;
     int M, N, K;
     int num_kb, splits, m_tiles, BN, stages;
+    int pair;                       // 1: columns j and j + BN/2 of the accumulator belong to the same token
     unsigned long long* argmax;
     float* logits;
     int* status;
@@ -60,7 +66,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     const int kb_end = (int)(((long long)a.num_kb * (split + 1)) / a.splits);
     const int n_kb = kb_end - kb_begin;
     const int f0 = out_tile * BM;       // first weight row (output feature) of the tile
-    const int m0 = m_tile * BN;         // first token row of the tile
+    const int m0 = m_tile * BN;         // first row of the tile in the activation buffer
+    const int TBk = a.pair ? BN / 2 : BN;   // tokens per tile
+    const int t0 = m_tile * TBk;        // first token of the tile
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t ncols = 32;
@@ -135,11 +143,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
         tc_fence_after();
         const int f = f0 + warp * 32 + lane;
         const bool f_ok = f < a.N;
-        for (int c = 0; c < BN / 16; ++c) {
+        for (int c = 0; c < TBk / 16; ++c) {
             uint32_t r[16];
             if (have) {
-                tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 16), r);
-                tmem_ld_wait();
+                const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+                tmem_ld16(lane_base + (uint32_t)(c * 16), r);
+                if (a.pair) {
+                    uint32_t r2[16];
+                    tmem_ld16(lane_base + (uint32_t)(TBk + c * 16), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                } else {
+                    tmem_ld_wait();
+                }
             } else {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) r[j] = 0u;
@@ -155,25 +172,25 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
                         const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
                         s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
                     }
-                    if (a.logits && f_ok && m0 + n < a.M) a.logits[(size_t)(m0 + n) * a.N + f] = __uint_as_float(r[j]);
+                    if (a.logits && f_ok && t0 + n < a.M) a.logits[(size_t)(t0 + n) * a.N + f] = __uint_as_float(r[j]);
                 }
             } else {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                    const int m = m0 + c * 16 + j;
+                    const int m = t0 + c * 16 + j;
                     if (f_ok && m < a.M) a.partials[((size_t)split * a.M + m) * a.N + f] = __uint_as_float(r[j]);
                 }
             }
         }
         if (a.argmax) {
             asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int n = threadIdx.x; n < BN; n += 128) {
-                if (m0 + n < a.M) {
+            for (int n = threadIdx.x; n < TBk; n += 128) {
+                if (t0 + n < a.M) {
                     unsigned long long best = s_arg[n];
                     best = max(best, s_arg[256 + n]);
                     best = max(best, s_arg[512 + n]);
                     best = max(best, s_arg[768 + n]);
-                    atomicMax(&a.argmax[m0 + n], best);
+                    atomicMax(&a.argmax[t0 + n], best);
                 }
             }
         }
@@ -221,12 +238,19 @@ tasc_status encode_tmap_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, u
     return r == CUDA_SUCCESS ? TASC_OK : TASC_ECUDA;
 }
 
-GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes) {
+int gemm_token_tile(int M, bool pair) {
+    const int cap = pair ? 128 : 256;                 // tokens per tile (UMMA N <= 256)
+    const int m_tiles = (M + cap - 1) / cap;
+    const int per = (M + m_tiles - 1) / m_tiles;
+    return std::max(16, (per + 15) / 16 * 16);
+}
+
+GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes, bool pair) {
     GemmPlan p;
-    p.m_tiles = (M + 255) / 256;
-    int per = (M + p.m_tiles - 1) / p.m_tiles;
-    p.BN = std::max(16, (per + 15) / 16 * 16);
-    p.m_tiles = (M + p.BN - 1) / p.BN;
+    p.pair = pair ? 1 : 0;
+    p.TB = gemm_token_tile(M, pair);
+    p.BN = pair ? 2 * p.TB : p.TB;
+    p.m_tiles = (M + p.TB - 1) / p.TB;
     p.out_tiles = (N + BM - 1) / BM;
     const int num_kb = (K + BK - 1) / BK;
     const int tiles = p.out_tiles * p.m_tiles;
@@ -258,7 +282,7 @@ tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, flo
     if (argmax && plan.splits != 1) return TASC_EINVAL;
     GemmArgs a;
     a.partials = partials; a.M = M; a.N = N; a.K = K;
-    a.num_kb = (K + BK - 1) / BK; a.splits = plan.splits; a.m_tiles = plan.m_tiles; a.BN = plan.BN; a.stages = plan.stages;
+    a.num_kb = (K + BK - 1) / BK; a.splits = plan.splits; a.m_tiles = plan.m_tiles; a.BN = plan.BN; a.stages = plan.stages; a.pair = plan.pair;
     a.argmax = argmax; a.logits = logits; a.status = status;
     const int grid = plan.out_tiles * plan.splits * plan.m_tiles;
     gemm_bf16_kernel<<<grid, GEMM_THREADS, plan.smem_bytes, stream>>>(*tmW, *tmX, a);

@@ -9,14 +9,17 @@ namespace tasc {
 // Computes partial sums P[s][m][n] = sum over the k-range of split s of X[m][k] * W[n][k]
 // (bf16 inputs, float32 accumulation in TMEM).  Consumers add the `splits` slices in order.
 struct GemmPlan {
-    int BN;          // token rows per CTA tile (UMMA N), multiple of 16, 16..256
-    int m_tiles;     // ceil(M / BN)
+    int pair;        // 1: activations are (hi, lo) bf16 row pairs, see gemm_tcgen05.cu
+    int TB;          // tokens per CTA tile, multiple of 16
+    int BN;          // activation rows per CTA tile (UMMA N) = TB, or 2 * TB in paired mode; 16..256
+    int m_tiles;     // ceil(M / TB)
     int out_tiles;   // ceil(N / 128): weight rows per CTA tile = UMMA M = 128
     int splits;      // split-K factor
     int stages;      // TMA -> MMA pipeline depth
     int smem_bytes;
 };
-GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes);
+GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes, bool pair);
+int gemm_token_tile(int M, bool pair);     // TB for M token rows
 inline size_t gemm_partial_bytes(const GemmPlan& p, int M, int N) { return (size_t)p.splits * M * N * sizeof(float); }
 
 // rows x cols bf16 row-major matrix, box = {64 cols, box_rows}, 128-byte swizzle.
@@ -51,20 +54,22 @@ void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t strid
 
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
-                       cudaStream_t stream);
+                       int TB, cudaStream_t stream);
 // x += sum_s P[s]; h = RMSNorm(x) * gain  (gain == null: only the residual update)
 template <typename T>
 void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,
-                          cudaStream_t stream);
-// qkv = sum_s P[s]; RoPE on q and k; q -> qbuf [M][n_q*hd]; k, v -> KV pages of the layer.
+                          int TB, cudaStream_t stream);
+// qkv = sum_s P[s]; RoPE on q and k; q -> qbuf [M][n_q*hd] (float32); k, v -> KV pages of the layer.
 template <typename T>
-void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp, const float2* rope, T* qbuf,
+void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp, const float2* rope, float* qbuf,
                             T* k_pages, T* v_pages, const int32_t* block_table, int max_pages, int page_size,
                             long long n_pages, int M, int R, int n_q, int n_kv, int hd, int max_positions, int* status,
                             cudaStream_t stream);
 // act = SiLU(gate) * up with gate = sum_s P[s][:, :dff], up = sum_s P[s][:, dff:]
 template <typename T>
-void launch_silu_mul(const float* partials, int splits, T* act, int M, int dff, cudaStream_t stream);
+void launch_silu_mul(const float* partials, int splits, T* act, int M, int dff, int TB, cudaStream_t stream);
+// float32 rows -> (hi, lo) bf16 row pairs in the tile-local layout of the paired GEMM
+void launch_split_rows(const float* x, __nv_bfloat16* buf, int M, int K, int TB, cudaStream_t stream);
 // y[M][N] = sum_s P[s]
 void launch_sum_partials(const float* partials, int splits, float* y, size_t n, cudaStream_t stream);
 void launch_fill_u64(unsigned long long* p, unsigned long long v, int n, cudaStream_t stream);
@@ -85,9 +90,9 @@ void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, 
 // ------------------------------------------------------------------ attention (attention.cu)
 // Verify attention of R query rows per sequence over the paged KV cache (grouped-query, causal within the rows).
 template <typename T>
-void launch_attention(const T* qbuf, const T* k_pages, const T* v_pages, const int32_t* block_table, int max_pages,
-                      int page_size, long long n_pages, const RowPlan& rp, T* out, float* scratch, int B, int R, int n_q,
-                      int n_kv, int hd, int n_splits, cudaStream_t stream);
+void launch_attention(const float* qbuf, const T* k_pages, const T* v_pages, const int32_t* block_table, int max_pages,
+                      int page_size, long long n_pages, const RowPlan& rp, T* out, int TB, float* scratch, int B, int R,
+                      int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream);
 size_t attention_scratch_bytes(int B, int R, int n_q, int hd, int n_splits);
 int attention_splits(int B, int n_kv, int max_ctx);
 

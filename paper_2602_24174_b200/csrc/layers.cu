@@ -67,7 +67,7 @@ __global__ void rows_prefill_kernel(RowPlan rp, const int32_t* tokens, int64_t s
 template <typename T>
 __global__ void __launch_bounds__(128)
 embed_norm_kernel(const T* __restrict__ embed, const int* __restrict__ row_tok, const float* __restrict__ gain, float eps,
-                  float* __restrict__ x, T* __restrict__ h, int d) {
+                  float* __restrict__ x, T* __restrict__ h, int d, int TB) {
     __shared__ float red[4];
     const int m = blockIdx.x;
     const T* e = embed + (size_t)row_tok[m] * d;
@@ -79,14 +79,14 @@ embed_norm_kernel(const T* __restrict__ embed, const int* __restrict__ row_tok, 
     }
     const float inv = 1.0f / sqrtf(block_sum(ss, red) / (float)d + eps);
     for (int j = threadIdx.x; j < d; j += blockDim.x)
-        h[(size_t)m * d + j] = Num<T>::from_f(x[(size_t)m * d + j] * inv * gain[j]);
+        ActStore<T>::put(h, m, j, d, TB, x[(size_t)m * d + j] * inv * gain[j]);
 }
 
 // x[m] += sum_s P[s][m]; h[m] = RMSNorm(x[m]) * gain
 template <typename T>
 __global__ void __launch_bounds__(128)
 residual_norm_kernel(const float* __restrict__ P, int splits, float* __restrict__ x, const float* __restrict__ gain,
-                     float eps, T* __restrict__ h, int M, int d) {
+                     float eps, T* __restrict__ h, int M, int d, int TB) {
     __shared__ float red[4];
     const int m = blockIdx.x;
     float ss = 0.f;
@@ -99,13 +99,13 @@ residual_norm_kernel(const float* __restrict__ P, int splits, float* __restrict_
     if (!gain) return;
     const float inv = 1.0f / sqrtf(block_sum(ss, red) / (float)d + eps);
     for (int j = threadIdx.x; j < d; j += blockDim.x)
-        h[(size_t)m * d + j] = Num<T>::from_f(x[(size_t)m * d + j] * inv * gain[j]);
+        ActStore<T>::put(h, m, j, d, TB, x[(size_t)m * d + j] * inv * gain[j]);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(128)
 qkv_rope_append_kernel(const float* __restrict__ P, int splits, RowPlan rp, const float2* __restrict__ rope,
-                       T* __restrict__ qbuf, T* __restrict__ k_pages, T* __restrict__ v_pages,
+                       float* __restrict__ qbuf, T* __restrict__ k_pages, T* __restrict__ v_pages,
                        const int32_t* __restrict__ block_table, int max_pages, int page_size, long long n_pages,
                        int M, int R, int n_q, int n_kv, int hd, int max_positions, int* status) {
     const int m = blockIdx.x;
@@ -114,7 +114,7 @@ qkv_rope_append_kernel(const float* __restrict__ P, int splits, RowPlan rp, cons
     const int qd = n_q * hd, kvd = n_kv * hd, N = qd + 2 * kvd;
     const int b = m / R;
     if (pos < 0) {
-        for (int j = threadIdx.x; j < qd; j += blockDim.x) qbuf[(size_t)m * qd + j] = Num<T>::from_f(0.f);
+        for (int j = threadIdx.x; j < qd; j += blockDim.x) qbuf[(size_t)m * qd + j] = 0.f;
         return;
     }
     bool kv_ok = true;
@@ -141,8 +141,8 @@ qkv_rope_append_kernel(const float* __restrict__ P, int splits, RowPlan rp, cons
         const float2 c = cs[i];
         const float ra = a * c.x - bb * c.y, rb = bb * c.x + a * c.y;
         if (head < n_q) {
-            qbuf[(size_t)m * qd + head * hd + i] = Num<T>::from_f(ra);
-            qbuf[(size_t)m * qd + head * hd + i + half] = Num<T>::from_f(rb);
+            qbuf[(size_t)m * qd + head * hd + i] = ra;
+            qbuf[(size_t)m * qd + head * hd + i + half] = rb;
         } else if (kv_ok) {
             const int kh = head - n_q;
             T* dst = k_pages + (((size_t)page * n_kv + kh) * page_size + slot) * hd;
@@ -159,7 +159,7 @@ qkv_rope_append_kernel(const float* __restrict__ P, int splits, RowPlan rp, cons
 }
 
 template <typename T>
-__global__ void silu_mul_kernel(const float* __restrict__ P, int splits, T* __restrict__ act, int M, int dff) {
+__global__ void silu_mul_kernel(const float* __restrict__ P, int splits, T* __restrict__ act, int M, int dff, int TB) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (size_t)M * dff) return;
     const int m = (int)(i / dff), j = (int)(i % dff);
@@ -169,7 +169,7 @@ __global__ void silu_mul_kernel(const float* __restrict__ P, int splits, T* __re
         g += row[j];
         u += row[dff + j];
     }
-    act[i] = Num<T>::from_f(g / (1.0f + expf(-g)) * u);
+    ActStore<T>::put(act, m, j, dff, TB, g / (1.0f + expf(-g)) * u);
 }
 
 __global__ void sum_partials_kernel(const float* __restrict__ P, int splits, float* __restrict__ y, size_t n) {
@@ -178,6 +178,12 @@ __global__ void sum_partials_kernel(const float* __restrict__ P, int splits, flo
     float v = 0.f;
     for (int s = 0; s < splits; ++s) v += P[(size_t)s * n + i];
     y[i] = v;
+}
+
+__global__ void split_rows_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ buf, int M, int K, int TB) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)M * K) return;
+    ActStore<__nv_bfloat16>::put(buf, (int)(i / K), (int)(i % K), K, TB, x[i]);
 }
 
 __global__ void fill_u64_kernel(unsigned long long* p, unsigned long long v, int n) {
@@ -273,16 +279,16 @@ void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t strid
 }
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
-                       cudaStream_t stream) {
-    embed_norm_kernel<T><<<M, 128, 0, stream>>>(embed, row_tok, gain, eps, x, h, d);
+                       int TB, cudaStream_t stream) {
+    embed_norm_kernel<T><<<M, 128, 0, stream>>>(embed, row_tok, gain, eps, x, h, d, TB);
 }
 template <typename T>
 void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,
-                          cudaStream_t stream) {
-    residual_norm_kernel<T><<<M, 128, 0, stream>>>(partials, splits, x, gain, eps, h, M, d);
+                          int TB, cudaStream_t stream) {
+    residual_norm_kernel<T><<<M, 128, 0, stream>>>(partials, splits, x, gain, eps, h, M, d, TB);
 }
 template <typename T>
-void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp, const float2* rope, T* qbuf,
+void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp, const float2* rope, float* qbuf,
                             T* k_pages, T* v_pages, const int32_t* block_table, int max_pages, int page_size,
                             long long n_pages, int M, int R, int n_q, int n_kv, int hd, int max_positions, int* status,
                             cudaStream_t stream) {
@@ -290,12 +296,16 @@ void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp
                                                      max_pages, page_size, n_pages, M, R, n_q, n_kv, hd, max_positions, status);
 }
 template <typename T>
-void launch_silu_mul(const float* partials, int splits, T* act, int M, int dff, cudaStream_t stream) {
+void launch_silu_mul(const float* partials, int splits, T* act, int M, int dff, int TB, cudaStream_t stream) {
     const size_t n = (size_t)M * dff;
-    silu_mul_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partials, splits, act, M, dff);
+    silu_mul_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partials, splits, act, M, dff, TB);
 }
 void launch_sum_partials(const float* partials, int splits, float* y, size_t n, cudaStream_t stream) {
     sum_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partials, splits, y, n);
+}
+void launch_split_rows(const float* x, __nv_bfloat16* buf, int M, int K, int TB, cudaStream_t stream) {
+    const size_t n = (size_t)M * K;
+    split_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(x, buf, M, K, TB);
 }
 void launch_fill_u64(unsigned long long* p, unsigned long long v, int n, cudaStream_t stream) {
     fill_u64_kernel<<<(n + 255) / 256, 256, 0, stream>>>(p, v, n);
@@ -328,12 +338,14 @@ void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, 
 }
 
 #define TASC_INSTANTIATE(T)                                                                                              \
-    template void launch_embed_norm<T>(const T*, const int*, const float*, float, float*, T*, int, int, cudaStream_t);   \
-    template void launch_residual_norm<T>(const float*, int, float*, const float*, float, T*, int, int, cudaStream_t);   \
-    template void launch_qkv_rope_append<T>(const float*, int, const RowPlan&, const float2*, T*, T*, T*,                \
+    template void launch_embed_norm<T>(const T*, const int*, const float*, float, float*, T*, int, int, int,             \
+                                       cudaStream_t);                                                                    \
+    template void launch_residual_norm<T>(const float*, int, float*, const float*, float, T*, int, int, int,             \
+                                          cudaStream_t);                                                                 \
+    template void launch_qkv_rope_append<T>(const float*, int, const RowPlan&, const float2*, float*, T*, T*,            \
                                             const int32_t*, int, int, long long, int, int, int, int, int, int, int*,     \
                                             cudaStream_t);                                                               \
-    template void launch_silu_mul<T>(const float*, int, T*, int, int, cudaStream_t);
+    template void launch_silu_mul<T>(const float*, int, T*, int, int, int, cudaStream_t);
 TASC_INSTANTIATE(float)
 TASC_INSTANTIATE(__nv_bfloat16)
 

@@ -52,3 +52,19 @@ def test_gemm_rejects_bad_arguments():
     w = torch.zeros((8, 60), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(b.TascError):
         b.tasc_gemm_bf16(x, w)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,N,K", [(6, 1152, 896), (7, 200, 72), (96, 960, 576), (130, 256, 4864), (300, 384, 256)])
+def test_paired_gemm_keeps_float32_activations(M, N, K):
+    """float32 X carried as (hi, lo) bf16 pairs: the error must be far below a plain bf16 rounding of X."""
+    b = need_gpu()
+    x = rng.normal(3, 1, 0, M * K, 1.0).reshape(M, K)                       # not bf16-representable
+    w = round_to_bf16(rng.normal(3, 2, 0, N * K, 0.05)).reshape(N, K)
+    y = b.tasc_gemm_bf16x2(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda().bfloat16()).cpu().numpy()
+    ref = linear(x.astype(np.float64), w.astype(np.float64))
+    err = np.abs(y - ref).max()
+    err_if_rounded = np.abs(linear(round_to_bf16(x).astype(np.float64), w.astype(np.float64)) - ref).max()
+    # hi + lo keeps 16 mantissa bits of x: error 2^-17 relative per term instead of 2^-9
+    assert err <= 3e-5 * np.sqrt(K) * np.abs(w).max() * np.abs(x).max() + 1e-6, err
+    assert err < err_if_rounded / 30

@@ -119,3 +119,41 @@ def test_verify_rejects_bad_arguments():
     ws = s.model.new_workspace(1, 4)
     with pytest.raises(b.TascError):
         b.tasc_verify_step(s.model, kv, seqs, torch.zeros((1, 16), dtype=torch.int32, device="cuda"), ws)   # k + 1 > 16
+
+
+# ------------------------------------------------------------------------------------------ bf16 configurations
+@pytest.fixture(scope="module")
+def setup1():
+    return make_setup(configs.get(1))
+
+
+@pytest.mark.gpu
+def test_config1_lockstep_batch1_full(setup1):
+    cfg = configs.get(1)
+    prompts = corpus.make_prompts(cfg, 1)
+    check(lockstep(setup1, prompts, cfg.max_new, cfg.k, **BF16_TOL))
+
+
+@pytest.mark.gpu
+def test_config1_lockstep_batch16_short(setup1):
+    cfg = configs.get(1)
+    prompts = corpus.make_prompts(cfg, 16)
+    check(lockstep(setup1, prompts, 12, cfg.k, **BF16_TOL))
+
+
+@pytest.mark.gpu
+def test_config1_teacher_forced_continuation(setup1):
+    cfg = configs.get(1)
+    prompts = corpus.make_prompts(cfg, 2)
+    cont = corpus.make_continuations(cfg, prompts, 40 + cfg.k + 1)
+    rep = lockstep(setup1, prompts, 40, cfg.k, oracle_kwargs=[dict(continuation=cont[i]) for i in range(2)],
+                   forced_mode="continuation", **BF16_TOL)
+    check(rep)
+
+
+@pytest.mark.gpu
+def test_config2_lockstep_short():
+    cfg = configs.get(2)
+    s = make_setup(cfg, n_docs=20000)
+    prompts = corpus.make_prompts(cfg, 2)
+    check(lockstep(s, prompts, 18, 8, **BF16_TOL))
