@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-decoding hot path: one step = draft k tokens per sequence (n-gram
+drafter) + verify the k+1 rows in one forward + greedy accept/commit, for one batch.
+
+    python bench.py --gpus 1 --steps 64 --warmup 8
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference          (the CPU oracle on a bounded sample of the same workload)
+
+Prints ONE JSON line.  Workload: configuration 1 (SLM-135M shape, bf16) at batch 16, k = 5, prompts of
+256 tokens, synthetic corpus / prompts / random-init weights.  `value` = tokens committed by all
+sequences on all ranks per second of device time over the K timed steps (prefill excluded, inputs
+resident in HBM); `e2e` = the same with the step's token buffers copied from pinned host memory and
+the results read back inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workload import configs, corpus, weights as W  # noqa: E402
+
+METRIC = "generated tokens/s with n-gram spec decode @1 B200; verify-step HBM GB/s vs peak"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"], "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback (earlier measurement on this pool)"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, smax, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax = float(f[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def step_bytes(shape, B, k, ctx_lens):
+    """Algorithmic HBM bytes of one verify step: every weight once, every live KV byte once, the new KV rows."""
+    wbytes = shape.matmul_params() * 2
+    kv = sum(ctx_lens) * shape.kv_bytes_per_token() + B * (k + 1) * shape.kv_bytes_per_token()
+    return wbytes, kv
+
+
+def gemm_bytes_per_step(shape, M):
+    """Algorithmic bytes of all GEMM launches of one step: weights + (hi, lo) activation rows in + float32 rows out."""
+    s = shape
+    mats = [(s.qkv_rows, s.d_model), (s.d_model, s.q_dim), (2 * s.d_ff, s.d_model), (s.d_model, s.d_ff)]
+    total = 0
+    for n, kk in mats:
+        total += s.n_layers * (n * kk * 2 + 2 * M * kk * 2 + M * n * 4)
+    total += s.vocab * s.d_model * 2 + 2 * M * s.d_model * 2          # LM head: argmax epilogue writes no logits
+    return total
+
+
+# ----------------------------------------------------------------------------------------------- oracle legs
+def oracle_sample(cfg, B_sample, n_steps, k, prompts):
+    """Times the CPU oracle (as it stands) on a bounded sample: B_sample sequences, prompt prefilled,
+    n_steps speculative steps each.  Returns (tokens/s over the decode steps, threads used, description)."""
+    from oracle import decode as G, drafter as D
+    from oracle.model import OracleModel
+    tokens, offsets = corpus.make_corpus(cfg, n_docs=min(cfg.corpus.n_docs, 20000))
+    ng = D.build_corpus_ngrams_sorted(tokens, offsets, cfg.n_max, cfg.p_min, cfg.model.vocab)
+    om = OracleModel(cfg.model, W.make_weights(cfg.model, cfg.seed_weights), np.float32)
+    committed_total, t_total = 0, 0.0
+    for i in range(B_sample):
+        committed = list(map(int, prompts[i]))
+        cache = om.new_cache(len(committed) + n_steps * (k + 1) + k + 2)
+        om.prefill(committed[:-1], cache)
+        t0 = time.perf_counter()
+        for _ in range(n_steps):
+            drafts = D.draft(ng, committed, k, cfg.lambda_num, cfg.lambda_den)
+            st = G.verify_step(om, cache, committed[-1], drafts)
+            committed += st.drafts[:st.n_accepted] + [st.next_token]
+            committed_total += st.n_accepted + 1
+        t_total += time.perf_counter() - t0
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        pass
+    desc = (f"config {cfg.index} ({cfg.name}): {B_sample} of the batch's sequences, prompt {cfg.prompt_len} prefilled "
+            f"(untimed), {n_steps} speculative steps each (k={k}), numpy float32, corpus tables from 20000 docs")
+    return committed_total / t_total, cores, desc, t_total / (B_sample * n_steps)
+
+
+def run_reference(args, cfg, B, k):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    prompts = corpus.make_prompts(cfg, 2)
+    # warm-up and timed steps are both bounded samples: 1 sequence, a few steps per "step"
+    n = max(1, min(args.steps, 16))
+    val, cores, desc, s_per_step = oracle_sample(cfg, 1, max(1, min(args.warmup, 2)) + n, k, prompts)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"config {cfg.index} ({cfg.name}) B={B} k={k} prompt {cfg.prompt_len}: bounded sample", "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------- device arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--batch", type=int, default=16)
+    ap.add_argument("--k", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only-timed", action="store_true",
+                    help="device-resident timed region only (no per-kernel pass, e2e, generate or CPU legs): the command ncu wraps")
+    ap.add_argument("--sweep", action="store_true", help="also report the teacher-forced acceptance sweep (forced a = 0..k)")
+    args = ap.parse_args()
+    cfg = configs.get(args.config)
+    B = args.batch
+    k = args.k or cfg.k
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args, cfg, B, k)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2602_24174_b200 import binding as b      # raises if libtasc.so is missing: there is no fallback
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    shape = cfg.model
+
+    # ---- inputs (seeded, synthetic); every rank is an independent replica with its own prompts
+    host_w = W.make_weights(shape, cfg.seed_weights)
+    model = b.Model(shape, b.weights_to_device(host_w, shape.dtype, dev), max_positions=cfg.prompt_len + cfg.max_new + 4096,
+                    page_size=cfg.page_size)
+    del host_w
+    ctoks, coffs = corpus.make_corpus(cfg)
+    drafter = b.tasc_drafter_build(torch.from_numpy(ctoks).to(dev), torch.from_numpy(coffs).to(dev), cfg.n_max, cfg.p_min, shape.vocab)
+    prompts_all = corpus.make_prompts(cfg, B * world)
+    prompts = prompts_all[rank * B:(rank + 1) * B]
+    P = prompts.shape[1]
+    total_steps = args.warmup + args.steps
+    stride = P + (total_steps + args.steps + 2) * (k + 1) + k + 2       # timed pass + instrumented pass share one state
+    if stride > 12288:
+        raise SystemExit("too many steps for one token buffer")
+    ws = model.new_workspace(B, k, dev)
+
+    def fresh_state():
+        tokens = torch.zeros((B, stride), dtype=torch.int32, device=dev)
+        tokens[:, :P] = torch.from_numpy(prompts).to(dev)
+        length = torch.full((B,), P, dtype=torch.int32, device=dev)
+        pool, bt, kv = model.new_kv(B, stride + b.MAX_ROWS, dev)
+        seqs = b.make_seqs(tokens, length)
+        b.tasc_prefill(model, kv, seqs, B, P, ws)
+        return tokens, length, (pool, bt, kv), seqs
+
+    drafts = torch.empty((B, k), dtype=torch.int32, device=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    def one_step(kvs, seqs, tokens, length):
+        b.tasc_draft(drafter, tokens, length, k, cfg.lambda_num, cfg.lambda_den, out=drafts)
+        return b.tasc_verify_step(model, kvs[2], seqs, drafts, ws)
+
+    # ---- device-resident timing: `value`
+    tokens, length, kvs, seqs = fresh_state()
+    for _ in range(args.warmup):
+        one_step(kvs, seqs, tokens, length)
+    b.tasc_poll_status(ws)
+    len0 = length.clone()
+    launches0 = sum(b.tasc_launch_counts().values())
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        one_step(kvs, seqs, tokens, length)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = sum(b.tasc_launch_counts().values()) - launches0
+    b.tasc_poll_status(ws)
+    ms = max_over_ranks(ev0.elapsed_time(ev1))
+    committed = float((length - len0).sum().item())
+    committed_all = sum_over_ranks(committed)
+    value = committed_all / (ms * 1e-3)
+    ctx_mid = (len0.float().mean().item() + length.float().mean().item()) / 2
+
+    if args.only_timed:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms / args.steps, "steps": args.steps,
+                              "warmup": args.warmup, "gpu_launches": int(launches), "only_timed": True}), flush=True)
+        return
+
+    # ---- per-kernel timing of the same steps in a separate, instrumented pass (events around every launch)
+    b.tasc_profile_enable(True)
+    b.tasc_profile_read()
+    for _ in range(args.steps):
+        one_step(kvs, seqs, tokens, length)
+    prof = b.tasc_profile_read()
+    b.tasc_profile_enable(False)
+    peaks = load_peaks()
+    M = B * (k + 1)
+    gemm_ms = prof["gemm"][0] + prof["gemm_lm_head_argmax"][0]
+    gemm_launches = prof["gemm"][1] + prof["gemm_lm_head_argmax"][1]
+    gemm_bytes = gemm_bytes_per_step(shape, M) * args.steps
+    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+    wbytes, kvbytes = step_bytes(shape, B, k, [ctx_mid] * B)
+    step_gbs = (wbytes + kvbytes) / (ms / args.steps * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": "gemm_bf16_kernel (tcgen05 + TMA; all projection, MLP and LM-head launches)",
+        "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+        "traffic": None, "peak_source": peaks["source"],
+        "bytes_per_launch_avg": gemm_bytes / max(gemm_launches, 1), "us_per_launch_avg": gemm_ms * 1e3 / max(gemm_launches, 1),
+        "launches": gemm_launches,
+        "verify_step": {"bytes_per_step": wbytes + kvbytes, "weight_bytes": wbytes, "kv_bytes": kvbytes,
+                        "achieved_gbs": step_gbs, "frac_of_measured_peak": step_gbs / peaks["hbm_gbs"],
+                        "frac_of_nominal_8000": step_gbs / 8000.0},
+        "kernel_ms_share": {kname: round(v[0] / max(sum(x[0] for x in prof.values()), 1e-9), 4) for kname, v in prof.items() if v[1]},
+    }
+
+    # ---- end to end: host token buffers in pinned memory, copied in and results copied out every step
+    tokens, length, kvs, seqs = fresh_state()
+    h_tokens = torch.zeros((B, stride), dtype=torch.int32).pin_memory()
+    h_tokens[:, :P] = torch.from_numpy(prompts)
+    h_len = torch.full((B,), P, dtype=torch.int32).pin_memory()
+    h_acc = torch.zeros(B, dtype=torch.int32).pin_memory()
+    h_next = torch.zeros(B, dtype=torch.int32).pin_memory()
+    h_drafts = torch.zeros((B, k), dtype=torch.int32).pin_memory()
+
+    def e2e_step():
+        tokens.copy_(h_tokens, non_blocking=True)
+        length.copy_(h_len, non_blocking=True)
+        n_acc, nxt, _, _ = one_step(kvs, seqs, tokens, length)
+        h_acc.copy_(n_acc, non_blocking=True)
+        h_next.copy_(nxt, non_blocking=True)
+        h_drafts.copy_(drafts, non_blocking=True)
+        torch.cuda.synchronize()
+        for i in range(B):                       # host-side commit of the step's result
+            L, a = int(h_len[i]), int(h_acc[i])
+            h_tokens[i, L:L + a] = h_drafts[i, :a]
+            h_tokens[i, L + a] = h_next[i]
+            h_len[i] = L + a + 1
+
+    for _ in range(args.warmup):
+        e2e_step()
+    len0_h = h_len.clone()
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    ms_e2e = max_over_ranks(ev0.elapsed_time(ev1))
+    e2e_val = sum_over_ranks(float((h_len - len0_h).sum().item())) / (ms_e2e * 1e-3)
+    e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h_tokens.numel() * 4 + h_len.numel() * 4),
+           "d2h_bytes_per_step": int((h_acc.numel() + h_next.numel() + h_drafts.numel()) * 4)}
+
+    # ---- whole-loop generation through tasc_generate (prefill + decode, device-side loop control)
+    gen = {}
+    if rank == 0:
+        def run_generate(mode, forced_accept=0, cont=None, max_new=cfg.max_new):
+            gstride = P + max_new + k + 2
+            gt = torch.zeros((B, gstride), dtype=torch.int32, device=dev)
+            gt[:, :P] = torch.from_numpy(prompts).to(dev)
+            gl = torch.full((B,), P, dtype=torch.int32, device=dev)
+            gpool, gbt, gkv = model.new_kv(B, gstride + b.MAX_ROWS, dev)
+            _, st = b.tasc_generate(model, drafter, gkv, b.make_seqs(gt, gl), B, max_new, k, ws, lambda_num=cfg.lambda_num,
+                                    lambda_den=cfg.lambda_den, mode=mode, forced_accept=forced_accept, continuation=cont)
+            hist = list(st.accepted_hist)[:k + 1]
+            seq_steps = max(sum(hist), 1)
+            return {"tokens_per_s": B * max_new / (st.decode_ms * 1e-3), "decode_ms": st.decode_ms, "prefill_ms": st.prefill_ms,
+                    "steps": st.steps, "mean_committed_per_step": st.committed / seq_steps, "accepted_hist": hist}
+        gen["greedy"] = run_generate(b.MODE_GREEDY)
+        cont = torch.from_numpy(corpus.make_continuations(cfg, prompts, cfg.max_new + k + 1)).to(dev)
+        gen["teacher_forced_continuation"] = run_generate(b.MODE_CONTINUATION, cont=cont)
+        if args.sweep:
+            gen["forced_accept_sweep"] = {str(a): run_generate(b.MODE_FORCED_ACCEPT, forced_accept=a) for a in range(k + 1)}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, desc, _ = oracle_sample(cfg, 2, 12, k, prompts_all[:2])
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if shape.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": f"config {cfg.index} ({cfg.name}): B={B} per GPU, k={k}, n_max={cfg.n_max}, prompt {P}, "
+                                   f"context {int(len0.float().mean().item())}->{int(length.float().mean().item())}, real greedy targets",
+                       "l2": "inputs larger than L2: weights %.0f MB are streamed once per step" % (wbytes / 1e6),
+                       "parallelism": "replicas only (independent batches per GPU, no collective)" if world > 1 else "single GPU"},
+            "mean_committed_per_step": committed_all / (args.steps * B * world),
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "generate": gen,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -252,6 +252,20 @@ tasc_status tasc_gemm_bf16x2(const float* x, const void* w, float* y, int32_t M,
                              void* workspace, size_t workspace_bytes, tasc_stream stream);
 size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
 
+/*
+ * Launch accounting.  Kernel launches are counted per kind for the life of the process
+ * (tasc_launch_counts).  With timing enabled, every launch is additionally bracketed by CUDA events
+ * on its own stream; tasc_profile_read synchronises the device, returns the summed milliseconds and
+ * the number of timed launches per kind since the last read, and forgets them.  Timing adds event
+ * records between kernels, so it belongs in a separate, untimed pass.
+ *   arrays: host, n >= tasc_profile_kinds() elements.
+ */
+int32_t     tasc_profile_kinds(void);
+const char* tasc_profile_kind_name(int32_t kind);
+tasc_status tasc_profile_enable(int32_t on);
+tasc_status tasc_profile_read(double* ms_by_kind, int64_t* timed_launches_by_kind, int32_t n);
+tasc_status tasc_launch_counts(int64_t* launches_by_kind, int32_t n);
+
 const char* tasc_status_string(tasc_status s);
 
 #ifdef __cplusplus

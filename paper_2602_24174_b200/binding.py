@@ -95,6 +95,17 @@ for _f in ("tasc_drafter_build", "tasc_drafter_export", "tasc_drafter_destroy", 
     getattr(lib, _f).restype = C.c_int32
 
 
+lib.tasc_profile_kinds.restype = C.c_int32
+lib.tasc_profile_kind_name.restype = C.c_char_p
+lib.tasc_profile_kind_name.argtypes = [C.c_int32]
+lib.tasc_profile_enable.argtypes = [C.c_int32]
+lib.tasc_profile_enable.restype = C.c_int32
+lib.tasc_profile_read.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64), C.c_int32]
+lib.tasc_profile_read.restype = C.c_int32
+lib.tasc_launch_counts.argtypes = [C.POINTER(C.c_int64), C.c_int32]
+lib.tasc_launch_counts.restype = C.c_int32
+
+
 def _check(code: int, where: str):
     if code != OK:
         raise TascError(code, where)
@@ -301,3 +312,27 @@ def weights_to_device(w: dict, dtype: str, device="cuda") -> dict:
     for lw in w["layers"]:
         out["layers"].append({k: conv(v, torch.float32 if k.endswith("norm") else td) for k, v in lw.items()})
     return out
+
+
+def profile_kinds():
+    return [lib.tasc_profile_kind_name(i).decode() for i in range(lib.tasc_profile_kinds())]
+
+
+def tasc_profile_enable(on: bool):
+    _check(lib.tasc_profile_enable(1 if on else 0), "tasc_profile_enable")
+
+
+def tasc_profile_read() -> dict:
+    """{kind: (milliseconds, timed launches)} since the last read."""
+    n = lib.tasc_profile_kinds()
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _check(lib.tasc_profile_read(ms, cnt, n), "tasc_profile_read")
+    return {k: (ms[i], cnt[i]) for i, k in enumerate(profile_kinds())}
+
+
+def tasc_launch_counts() -> dict:
+    n = lib.tasc_profile_kinds()
+    cnt = (C.c_int64 * n)()
+    _check(lib.tasc_launch_counts(cnt, n), "tasc_launch_counts")
+    return {k: cnt[i] for i, k in enumerate(profile_kinds())}

@@ -215,7 +215,11 @@ void launch_attention(const float* qbuf, const T* k_pages, const T* v_pages, con
         cudaFuncSetAttribute(attention_split_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         done = true;
     }
-    attention_split_kernel<T><<<dim3(n_splits, n_kv, B), ATT_THREADS, smem, stream>>>(a);
+    {
+        ProfScope ps(K_ATT_SPLIT, stream);
+        attention_split_kernel<T><<<dim3(n_splits, n_kv, B), ATT_THREADS, smem, stream>>>(a);
+    }
+    ProfScope ps(K_ATT_COMBINE, stream);
     attention_combine_kernel<T><<<dim3(R, n_q, B), hd < 128 ? 64 : 128, 0, stream>>>(a.o_part, a.ml_part, rp, out, TB, R, n_q, hd, n_splits);
 }
 

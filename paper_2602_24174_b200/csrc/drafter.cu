@@ -574,6 +574,7 @@ extern "C" tasc_status tasc_draft(const tasc_drafter* d, const int32_t* tokens, 
         TASC_CUDA_TRY(cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         attr = true;
     }
+    ProfScope ps(K_DRAFT, static_cast<cudaStream_t>(stream));
     draft_kernel<<<B, DRAFT_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(
         d->dt, tokens, stride, len, k, (uint32_t)lambda_num, (uint32_t)lambda_den, drafts, (int)(hs - 1));
     TASC_CUDA_TRY(cudaGetLastError());

@@ -44,6 +44,7 @@ gemm_f32_kernel(const float* __restrict__ X, const float* __restrict__ W, float*
 
 void launch_gemm_f32(const float* X, const float* W, float* partials, int M, int N, int K,
                      unsigned long long* argmax, float* logits, cudaStream_t stream) {
+    ProfScope ps(argmax ? K_GEMM_LM : K_GEMM, stream);
     dim3 grid((N + 3) / 4, (M + ROWS - 1) / ROWS);
     gemm_f32_kernel<<<grid, 128, 0, stream>>>(X, W, partials, M, N, K, argmax, logits);
 }

@@ -285,6 +285,7 @@ tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, flo
     a.num_kb = (K + BK - 1) / BK; a.splits = plan.splits; a.m_tiles = plan.m_tiles; a.BN = plan.BN; a.stages = plan.stages; a.pair = plan.pair;
     a.argmax = argmax; a.logits = logits; a.status = status;
     const int grid = plan.out_tiles * plan.splits * plan.m_tiles;
+    ProfScope ps(argmax ? K_GEMM_LM : K_GEMM, stream);
     gemm_bf16_kernel<<<grid, GEMM_THREADS, plan.smem_bytes, stream>>>(*tmW, *tmX, a);
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;

@@ -5,6 +5,17 @@
 
 namespace tasc {
 
+// ------------------------------------------------------------------ launch accounting (profile.cu)
+enum Kind { K_DRAFT, K_ROWS, K_EMBED, K_GEMM, K_GEMM_LM, K_QKV_ROPE, K_ATT_SPLIT, K_ATT_COMBINE, K_RESNORM, K_SILU,
+            K_ACCEPT, K_OTHER, K_COUNT };
+void prof_begin(int kind, cudaStream_t s);     // counts the launch; records an event when timing is enabled
+void prof_end(int kind, cudaStream_t s);
+struct ProfScope {
+    int kind; cudaStream_t s;
+    ProfScope(int k, cudaStream_t st) : kind(k), s(st) { prof_begin(kind, s); }
+    ~ProfScope() { prof_end(kind, s); }
+};
+
 // ------------------------------------------------------------------ tensor-core GEMM (gemm_tcgen05.cu)
 // Computes partial sums P[s][m][n] = sum over the k-range of split s of X[m][k] * W[n][k]
 // (bf16 inputs, float32 accumulation in TMEM).  Consumers add the `splits` slices in order.

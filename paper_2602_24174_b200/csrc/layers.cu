@@ -271,20 +271,24 @@ __global__ void min_generated_kernel(const int32_t* len, const int32_t* prompt_l
 void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len,
                         const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
                         cudaStream_t stream) {
+    ProfScope ps(K_ROWS, stream);
     rows_verify_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, stop_len, drafts, B, R, vocab, status);
 }
 void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
                          int chunk, int vocab, int* status, cudaStream_t stream) {
+    ProfScope ps(K_ROWS, stream);
     rows_prefill_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, B, R, chunk, vocab, status);
 }
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
                        int TB, cudaStream_t stream) {
+    ProfScope ps(K_EMBED, stream);
     embed_norm_kernel<T><<<M, 128, 0, stream>>>(embed, row_tok, gain, eps, x, h, d, TB);
 }
 template <typename T>
 void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,
                           int TB, cudaStream_t stream) {
+    ProfScope ps(K_RESNORM, stream);
     residual_norm_kernel<T><<<M, 128, 0, stream>>>(partials, splits, x, gain, eps, h, M, d, TB);
 }
 template <typename T>
@@ -292,48 +296,58 @@ void launch_qkv_rope_append(const float* partials, int splits, const RowPlan& rp
                             T* k_pages, T* v_pages, const int32_t* block_table, int max_pages, int page_size,
                             long long n_pages, int M, int R, int n_q, int n_kv, int hd, int max_positions, int* status,
                             cudaStream_t stream) {
+    ProfScope ps(K_QKV_ROPE, stream);
     qkv_rope_append_kernel<T><<<M, 128, 0, stream>>>(partials, splits, rp, rope, qbuf, k_pages, v_pages, block_table,
                                                      max_pages, page_size, n_pages, M, R, n_q, n_kv, hd, max_positions, status);
 }
 template <typename T>
 void launch_silu_mul(const float* partials, int splits, T* act, int M, int dff, int TB, cudaStream_t stream) {
+    ProfScope ps(K_SILU, stream);
     const size_t n = (size_t)M * dff;
     silu_mul_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partials, splits, act, M, dff, TB);
 }
 void launch_sum_partials(const float* partials, int splits, float* y, size_t n, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     sum_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(partials, splits, y, n);
 }
 void launch_split_rows(const float* x, __nv_bfloat16* buf, int M, int K, int TB, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     const size_t n = (size_t)M * K;
     split_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(x, buf, M, K, TB);
 }
 void launch_fill_u64(unsigned long long* p, unsigned long long v, int n, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     fill_u64_kernel<<<(n + 255) / 256, 256, 0, stream>>>(p, v, n);
 }
 void launch_accept(const unsigned long long* argmax, const RowPlan& rp, const int32_t* drafts,
                    const int32_t* forced_targets, int32_t* tokens, int64_t stride, int32_t* len, int B, int R,
                    int32_t* n_accepted, int32_t* next_token, int32_t* target_tokens, long long* hist,
                    cudaStream_t stream) {
+    ProfScope ps(K_ACCEPT, stream);
     accept_kernel<<<(B + 63) / 64, 64, 0, stream>>>(argmax, rp, drafts, forced_targets, tokens, stride, len, B, R,
                                                     n_accepted, next_token, target_tokens, hist);
 }
 void launch_rope_table(float2* table, int max_positions, int hd, float base, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     const int n = max_positions * (hd / 2);
     rope_table_kernel<<<(n + 255) / 256, 256, 0, stream>>>(table, max_positions, hd, base);
 }
 void launch_forced_targets(int mode, const int32_t* drafts, const int32_t* continuation, int64_t cont_stride,
                            const int32_t* len, const int32_t* prompt_len, int forced_accept, int vocab, int B, int k,
                            int32_t* targets, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     const int n = B * (k + 1);
     forced_targets_kernel<<<(n + 127) / 128, 128, 0, stream>>>(mode, drafts, continuation, cont_stride, len, prompt_len,
                                                                forced_accept, vocab, B, k, targets);
 }
 void launch_gather_output(const int32_t* tokens, int64_t stride, const int32_t* prompt_len, int B, int max_new,
                           int32_t* out, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     const int n = B * max_new;
     gather_output_kernel<<<(n + 255) / 256, 256, 0, stream>>>(tokens, stride, prompt_len, B, max_new, out);
 }
 void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, int* out_min, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
     min_generated_kernel<<<1, 128, 0, stream>>>(len, prompt_len, B, out_min);
 }
 
