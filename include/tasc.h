@@ -253,6 +253,35 @@ tasc_status tasc_gemm_bf16x2(const float* x, const void* w, float* y, int32_t M,
 size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
 
 /*
+ * The product of tasc_gemm_bf16 for callers that cannot allocate.  (The paper has no counterpart: this is
+ * a service entry point of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where device memory can no longer be requested -- inside a serving process
+ * whose memory pool was fixed at start-up, under a host that forbids cudaMalloc once initialisation is over,
+ * or anywhere no allocator is at hand to provide the split-K workspace that tasc_gemm_bf16 demands.  Here
+ * the partial sums go to a fixed 8 MiB device array that is part of the library image, so every GPU that
+ * loads the library holds those 8 MiB until the process exits.  The call itself requests no memory of any
+ * kind (no cudaMalloc / cudaFree, no allocating library routine); the caller passes inputs and output.
+ * (If launch timing was switched on with tasc_profile_enable, the accounting creates CUDA events as usual.)
+ *
+ *   x, w, y, M, N, K   as tasc_gemm_bf16
+ *   device_status      device, int32, or NULL: receives a device-side error code of this call (0 = none),
+ *                      cleared at the start of the call; with NULL the word lives inside the shared array
+ * Limits and rules:
+ *   - the float32 partial sums (k-splits * M * N * 4 bytes) must fit in 8 MiB minus 256 bytes; the call takes
+ *     fewer k-splits than tasc_gemm_bf16 if that makes them fit (only the summation order changes) and
+ *     returns TASC_ECAPACITY when even one split does not (M * N * 4 > 8 MiB - 256);
+ *   - the first call on each device looks up the array's device address (that device must be current, as
+ *     for every call) -- make that first call before starting any stream capture;
+ *   - all calls share the array and it keeps the previous call's contents; the kernel overwrites everything
+ *     it later reads, so calls that follow each other on one stream are safe, but calls that overlap on the
+ *     GPU (different streams or threads) race on it and corrupt each other's results.
+ * Asynchronous on the stream.  Errors: EINVAL, ECAPACITY, ECUDA.
+ */
+tasc_status tasc_gemm_bf16_static(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                                  int32_t* device_status, tasc_stream stream);
+
+/*
  * Launch accounting.  Kernel launches are counted per kind for the life of the process
  * (tasc_launch_counts).  With timing enabled, every launch is additionally bracketed by CUDA events
  * on its own stream; tasc_profile_read synchronises the device, returns the summed milliseconds and

@@ -88,6 +88,8 @@ lib.tasc_poll_status.argtypes = [_P, _P]
 lib.tasc_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 lib.tasc_gemm_bf16x2.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 lib.tasc_gemm_bf16x2.restype = C.c_int32
+lib.tasc_gemm_bf16_static.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, _P]
+lib.tasc_gemm_bf16_static.restype = C.c_int32
 lib.tasc_gemm_workspace_bytes.restype = C.c_size_t
 lib.tasc_gemm_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
 for _f in ("tasc_drafter_build", "tasc_drafter_export", "tasc_drafter_destroy", "tasc_draft", "tasc_model_create",
@@ -300,6 +302,26 @@ def tasc_gemm_bf16x2(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
     y = torch.empty((M, N), dtype=torch.float32, device=x.device)
     _check(lib.tasc_gemm_bf16x2(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(ws), ws.numel(), _stream()), "tasc_gemm_bf16x2")
     tasc_poll_status(ws)
+    return y
+
+
+def tasc_gemm_bf16_static(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, device_status: torch.Tensor | None = None):
+    """Y[M, N] float32 = X[M, K] @ W[N, K]^T for bf16 CUDA tensors, written into the caller's ``y``.
+
+    For callers that cannot allocate device memory: the split-K partial sums use the library's fixed
+    8 MiB device array, so this wrapper (unlike ``tasc_gemm_bf16``) creates no tensor either.
+    ``device_status``: optional int32[1] CUDA tensor that receives a device-side error code.  Raises
+    TascError(ECAPACITY) when M * N * 4 bytes exceed the array."""
+    _dev(x, torch.bfloat16)
+    _dev(w, torch.bfloat16)
+    _dev(y, torch.float32)
+    M, K = x.shape
+    N = w.shape[0]
+    assert tuple(y.shape) == (M, N)
+    if device_status is not None:
+        _dev(device_status, torch.int32)
+    _check(lib.tasc_gemm_bf16_static(_ptr(x), _ptr(w), _ptr(y), M, N, K, _ptr(device_status), _stream()),
+           "tasc_gemm_bf16_static")
     return y
 
 
