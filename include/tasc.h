@@ -296,6 +296,8 @@ tasc_status tasc_profile_read(double* ms_by_kind, int64_t* timed_launches_by_kin
 tasc_status tasc_launch_counts(int64_t* launches_by_kind, int32_t n);
 
 const char* tasc_status_string(tasc_status s);
+/* Text of the most recent failing CUDA runtime call behind a TASC_ECUDA (name, message, source location), or "". */
+const char* tasc_last_error(void);
 
 #ifdef __cplusplus
 }

@@ -31,7 +31,8 @@ MODE_GREEDY, MODE_CONTINUATION, MODE_FORCED_ACCEPT = 0, 1, 2
 class TascError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {lib.tasc_status_string(code).decode()} ({code})")
+        detail = lib.tasc_last_error().decode() if code == ECUDA else ""
+        super().__init__(f"{where}: {lib.tasc_status_string(code).decode()} ({code})" + (f": {detail}" if detail else ""))
 
 
 class NgramEntry(C.Structure):
@@ -71,6 +72,7 @@ class Stats(C.Structure):
 _P = C.c_void_p
 lib.tasc_status_string.restype = C.c_char_p
 lib.tasc_status_string.argtypes = [C.c_int32]
+lib.tasc_last_error.restype = C.c_char_p
 lib.tasc_drafter_build.argtypes = [_P, _P, C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(_P)]
 lib.tasc_drafter_export.argtypes = [_P, C.POINTER(NgramEntry), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 lib.tasc_drafter_destroy.argtypes = [_P]

@@ -15,7 +15,7 @@ struct tasc_model {
     std::vector<const float*> attn_norm, mlp_norm;
     std::vector<const void*> wqkv, wo, w_gate_up, w_down;
     float2* rope;                                   // [max_positions][head_dim / 2] (cos, sin), library-owned
-    // tensor maps of the weight matrices (bf16 models): box = 64 x 128
+    // tensor maps of the weight matrices (bf16 models): box = 64 columns x 128 rows (gate/up: 64 rows, see EPI_SWIGLU)
     std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
     CUtensorMap tm_lm;
     int qkv_rows, q_dim, kv_dim;
@@ -49,6 +49,9 @@ struct Workspace {
     float* partials;
     size_t partial_bytes;
     float* att_scratch;
+    float* ssq;                   // [M][ceil(d / 128)] partial sums of squares of the residual rows (bf16 models)
+    int ssq_slots;
+    unsigned int* counters;       // [B * n_kv] attention merge tickets
     size_t bytes;
 };
 
@@ -85,7 +88,13 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     w.partial_bytes = std::max(MIN_PARTIAL_BYTES, M * n_max * sizeof(float));
     w.partials = L.take<float>(base, w.partial_bytes / sizeof(float));
     const int splits_max = attention_splits(B, d.n_kv_heads, 1 << 30);
-    w.att_scratch = L.take<float>(base, attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max) / sizeof(float));
+    const size_t att_bytes = d.dtype == TASC_F32
+        ? attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max)
+        : attention_mma_scratch_bytes(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * TASC_MAX_ROWS, splits_max);
+    w.att_scratch = L.take<float>(base, att_bytes / sizeof(float));
+    w.ssq_slots = (d.d_model + 127) / 128;
+    w.ssq = L.take<float>(base, M * w.ssq_slots);
+    w.counters = L.take<unsigned int>(base, (size_t)B * d.n_kv_heads);
     w.bytes = L.off;
     return w;
 }
@@ -185,10 +194,80 @@ tasc_status forward(const tasc_model* m, const tasc_kv* kv, const Workspace& w, 
     return TASC_OK;
 }
 
+// bf16 models: five launches per layer (QKV+RoPE+KV append, attention, O+residual, gate/up+SiLU*mul, down+residual),
+// each with programmatic stream serialisation; see gemm_fused.cu and attention_mma.cu.
+tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
+                         cudaStream_t s) {
+    const tasc_model_desc& d = m->desc;
+    const int M = B * R;
+    const int max_ctx = kv->max_pages_per_seq * d.page_size;
+    const int att_splits = attention_splits(B, d.n_kv_heads, max_ctx);
+    const int TB = gemm_token_tile(M, true);
+    const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
+    CUtensorMap tm_h, tm_o, tm_act;
+    tasc_status st;
+    if ((st = encode_tmap_bf16(&tm_h, w.h, rows, d.d_model, 2 * TB)) != TASC_OK) return st;
+    if ((st = encode_tmap_bf16(&tm_o, w.o, rows, m->q_dim, 2 * TB)) != TASC_OK) return st;
+    if ((st = encode_tmap_bf16(&tm_act, w.act, rows, d.d_ff, 2 * TB)) != TASC_OK) return st;
+    const FusedPlan p_qkv = plan_fused(M, m->qkv_rows, d.d_model, EPI_QKV);
+    const FusedPlan p_o = plan_fused(M, d.d_model, m->q_dim, EPI_RESID);
+    const FusedPlan p_gu = plan_fused(M, d.d_ff, d.d_model, EPI_SWIGLU);
+    const FusedPlan p_down = plan_fused(M, d.d_model, d.d_ff, EPI_RESID);
+    __nv_bfloat16* h = static_cast<__nv_bfloat16*>(w.h);
+    __nv_bfloat16* o = static_cast<__nv_bfloat16*>(w.o);
+    __nv_bfloat16* act = static_cast<__nv_bfloat16*>(w.act);
+
+    FusedArgs base = {};
+    base.M = M;
+    base.ssq_slots = w.ssq_slots;
+    base.inv_d = 1.0f / (float)d.d_model;
+    base.eps = d.rms_eps;
+    base.status = w.status;
+
+    launch_embed_scaled(static_cast<const __nv_bfloat16*>(m->embed), w.rp.row_tok, m->attn_norm[0], w.x, h, w.ssq, w.ssq_slots,
+                        lm_head ? w.argmax : nullptr, M, d.d_model, TB, s);
+    for (int l = 0; l < d.n_layers; ++l) {
+        const KvView kvl = layer_kv(m, kv, l);
+        FusedArgs a = base;
+        a.N = m->qkv_rows; a.K = d.d_model; a.ssq_in = w.ssq;
+        a.row_pos = w.rp.row_pos; a.rope = m->rope; a.qbuf = w.q;
+        a.k_pages = static_cast<__nv_bfloat16*>(kvl.k); a.v_pages = static_cast<__nv_bfloat16*>(kvl.v);
+        a.block_table = kv->block_table; a.max_pages = kv->max_pages_per_seq; a.page_size = d.page_size; a.n_pages = kv->n_pages;
+        a.R = R; a.n_q = d.n_q_heads; a.n_kv = d.n_kv_heads; a.hd = d.head_dim; a.max_positions = d.max_positions;
+        if ((st = launch_gemm_fused(EPI_QKV, &m->tm_qkv[l], &tm_h, a, p_qkv, s)) != TASC_OK) return st;
+
+        st = launch_attention_mma(w.q, static_cast<const __nv_bfloat16*>(kvl.k), static_cast<const __nv_bfloat16*>(kvl.v),
+                                  kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, w.att_scratch,
+                                  w.counters, B, R, d.n_q_heads, d.n_kv_heads, d.head_dim, att_splits, s);
+        if (st != TASC_OK) return st;
+
+        a = base;
+        a.N = d.d_model; a.K = m->q_dim; a.x = w.x; a.gain = m->mlp_norm[l]; a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = w.ssq_slots;
+        if ((st = launch_gemm_fused(EPI_RESID, &m->tm_o[l], &tm_o, a, p_o, s)) != TASC_OK) return st;
+
+        a = base;
+        a.N = d.d_ff; a.K = d.d_model; a.ssq_in = w.ssq; a.a_out = act;
+        if ((st = launch_gemm_fused(EPI_SWIGLU, &m->tm_gu[l], &tm_h, a, p_gu, s)) != TASC_OK) return st;
+
+        a = base;
+        a.N = d.d_model; a.K = d.d_ff; a.x = w.x; a.gain = l + 1 < d.n_layers ? m->attn_norm[l + 1] : m->final_norm;
+        a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = w.ssq_slots;
+        if ((st = launch_gemm_fused(EPI_RESID, &m->tm_down[l], &tm_act, a, p_down, s)) != TASC_OK) return st;
+    }
+    if (lm_head) {
+        const FusedPlan p_lm = plan_fused(M, d.vocab, d.d_model, EPI_LM);
+        FusedArgs a = base;
+        a.N = d.vocab; a.K = d.d_model; a.ssq_in = w.ssq; a.argmax = w.argmax; a.logits = logits;
+        if ((st = launch_gemm_fused(EPI_LM, &m->tm_lm, &tm_h, a, p_lm, s)) != TASC_OK) return st;
+    }
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
 tasc_status forward_any(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
                         cudaStream_t s) {
     return m->desc.dtype == TASC_F32 ? forward<float>(m, kv, w, B, R, lm_head, logits, s)
-                                     : forward<__nv_bfloat16>(m, kv, w, B, R, lm_head, logits, s);
+                                     : forward_bf16(m, kv, w, B, R, lm_head, logits, s);
 }
 
 bool check_common(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, int B, void* ws, size_t ws_bytes) {
@@ -203,7 +282,8 @@ tasc_status verify_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_se
                            const int32_t* drafts, int B, int k, const int32_t* forced, int32_t* n_accepted,
                            int32_t* next_token, int32_t* target_tokens, float* logits, cudaStream_t s) {
     const int R = k + 1;
-    launch_rows_verify(w.rp, seqs->tokens, seqs->stride, seqs->len, seqs->stop_len, drafts, B, R, m->desc.vocab, w.status, s);
+    launch_rows_verify(w.rp, seqs->tokens, seqs->stride, seqs->len, seqs->stop_len, drafts, B, R, m->desc.vocab, w.status, w.counters,
+                       B * m->desc.n_kv_heads, s);
     tasc_status st = forward_any(m, kv, w, B, R, true, logits, s);
     if (st != TASC_OK) return st;
     launch_accept(w.argmax, w.rp, drafts, forced, seqs->tokens, seqs->stride, seqs->len, B, R, n_accepted, next_token,
@@ -217,7 +297,8 @@ tasc_status prefill_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_s
     const int R = TASC_MAX_ROWS;
     const int chunks = (std::max(max_len - 1, 0) + R - 1) / R;
     for (int c = 0; c < chunks; ++c) {
-        launch_rows_prefill(w.rp, seqs->tokens, seqs->stride, seqs->len, B, R, c, m->desc.vocab, w.status, s);
+        launch_rows_prefill(w.rp, seqs->tokens, seqs->stride, seqs->len, B, R, c, m->desc.vocab, w.status, w.counters,
+                            B * m->desc.n_kv_heads, s);
         tasc_status st = forward_any(m, kv, w, B, R, false, nullptr, s);
         if (st != TASC_OK) return st;
     }
@@ -242,6 +323,11 @@ extern "C" tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc
     if (!wt->embed || !wt->lm_head || !wt->final_norm || !wt->attn_norm || !wt->wqkv || !wt->wo || !wt->mlp_norm ||
         !wt->w_gate_up || !wt->w_down)
         return TASC_EINVAL;
+    if (d.dtype == TASC_BF16) {
+        // tensor-core attention: head_dim 32, 64 or 128 and at most 128 query rows per KV head in a prefill chunk
+        if (d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128) return TASC_EINVAL;
+        if ((d.n_q_heads / d.n_kv_heads) * TASC_MAX_ROWS > 128) return TASC_EINVAL;
+    }
     tasc_model* m = new (std::nothrow) tasc_model();
     if (!m) return TASC_ENOMEM;
     m->desc = d;
@@ -266,7 +352,7 @@ extern "C" tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc
         for (int l = 0; l < d.n_layers && st == TASC_OK; ++l) {
             st = encode_tmap_bf16(&m->tm_qkv[l], m->wqkv[l], m->qkv_rows, d.d_model, 128);
             if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_o[l], m->wo[l], d.d_model, m->q_dim, 128);
-            if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_gu[l], m->w_gate_up[l], 2 * (uint64_t)d.d_ff, d.d_model, 128);
+            if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_gu[l], m->w_gate_up[l], 2 * (uint64_t)d.d_ff, d.d_model, 64);
             if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_down[l], m->w_down[l], d.d_model, d.d_ff, 128);
         }
         if (st == TASC_OK) st = encode_tmap_bf16(&m->tm_lm, m->lm_head, d.vocab, d.d_model, 128);
@@ -444,22 +530,20 @@ extern "C" tasc_status tasc_gemm_bf16x2(const float* x, const void* wt, float* y
     if (reinterpret_cast<uintptr_t>(workspace) % 256) return TASC_EINVAL;
     if (workspace_bytes < tasc_gemm_workspace_bytes(M, N, K)) return TASC_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40, true);
-    tasc_status st = gemm_set_attributes();
-    if (st != TASC_OK) return st;
+    // the forward's kernel with the plain epilogue: split-K inside a cluster, no partial sums in global memory
+    const FusedPlan p = plan_fused(M, N, K, EPI_PLAIN);
     int* status = static_cast<int*>(workspace);
-    uint8_t* base = static_cast<uint8_t*>(workspace) + 256;
-    float* partials = reinterpret_cast<float*>(base);
-    const size_t pb = (gemm_partial_bytes(p, M, N) + 255) / 256 * 256;
-    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(base + pb);
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + 256);
     const uint64_t rows = (uint64_t)p.m_tiles * p.BN;
     TASC_CUDA_TRY(cudaMemsetAsync(xs, 0, rows * K * 2, s));
     launch_split_rows(x, xs, M, K, p.TB, s);
     CUtensorMap tmW, tmX;
+    tasc_status st;
     if ((st = encode_tmap_bf16(&tmW, wt, N, K, 128)) != TASC_OK) return st;
     if ((st = encode_tmap_bf16(&tmX, xs, rows, K, p.BN)) != TASC_OK) return st;
-    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, nullptr, nullptr, status, s)) != TASC_OK) return st;
-    launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
+    FusedArgs a = {};
+    a.M = M; a.N = N; a.K = K; a.y = y; a.status = status;
+    if ((st = launch_gemm_fused(EPI_PLAIN, &tmW, &tmX, a, p, s)) != TASC_OK) return st;
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;
 }

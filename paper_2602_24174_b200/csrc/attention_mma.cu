@@ -1,0 +1,399 @@
+// Verify attention for bf16 models on the warp-level tensor-core path: the R = k+1 new query rows of a
+// sequence times the g query heads that share one KV head (G = g * R rows) against the paged KV cache.
+//
+// The kernel is bound by streaming K and V from HBM once; the tensor cores only have to keep up with
+// that stream, which a float32 SIMT formulation cannot do beyond a few sequences.  A CTA owns one
+// (sequence, KV head, key range): the key range of a sequence is split over several CTAs because the
+// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a two-stage cp.async pipeline
+// (16-byte vectors, every page of a KV head is one contiguous run) into XOR-swizzled shared memory;
+// warp w computes the 16-row slab w of S = Q K^T and O += P V with mma.sync m16n8k16 (ldmatrix
+// fragments, V through ldmatrix.trans) and keeps an online softmax per row in registers.
+//
+// Precision: K and V are bf16 as stored.  Q (pre-scaled by log2(e) / sqrt(head_dim)) and the
+// probabilities P are float32 values carried as hi + lo bf16 pairs, two MMAs each, so the only rounding
+// in the attention is the KV cache's own.  Softmax statistics and O are float32.
+//
+// Merge: each CTA writes its unnormalised O and (max, sum) to scratch and takes a ticket; the CTA
+// that draws the last ticket of a (sequence, KV head) merges the splits in index order and writes the
+// result as (hi, lo) bf16 rows in the layout the O-projection GEMM loads.  Which CTA merges depends on
+// timing, what it computes does not.
+#include "kernels.h"
+
+namespace tasc {
+
+namespace {
+
+constexpr int TKEYS = 64;
+
+struct AttnArgs {
+    const float* q;                    // [M][n_q * hd], RoPE applied
+    const __nv_bfloat16* kp;
+    const __nv_bfloat16* vp;
+    const int32_t* block_table;
+    int max_pages, page_size;
+    long long n_pages;
+    const int* seq_pos0;
+    const int* seq_rows;
+    __nv_bfloat16* out;                // (hi, lo) activation buffer, row length n_q * hd
+    int TB;
+    float* o_part;                     // [B][n_kv][splits][GP][hd]
+    float2* ml_part;                   // [B][n_kv][splits][GP]
+    unsigned int* counters;            // [B][n_kv], zero between uses
+    int R, n_q, n_kv, splits;
+    float scale_log2e;
+};
+
+// Byte offset of 16-byte chunk `chunk` of row `row` in a [rows][HD] bf16 tile; the XOR keeps the eight
+// rows of an ldmatrix phase on distinct banks.
+template <int HD>
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+    constexpr int RB = HD * 2;
+    if (RB >= 128) return (uint32_t)(row * RB + ((chunk ^ (row & 7)) << 4));
+    return (uint32_t)(row * RB + ((chunk ^ ((row >> 1) & 3)) << 4));
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// two floats -> packed bf16 pair (hi) and the packed pair of the residuals (lo)
+__device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32_t& lo) {
+    __nv_bfloat16 hx, lx, hy, ly;
+    split_bf16(x, hx, lx);
+    split_bf16(y, hy, ly);
+    hi = (uint32_t)__bfloat16_as_ushort(hx) | ((uint32_t)__bfloat16_as_ushort(hy) << 16);
+    lo = (uint32_t)__bfloat16_as_ushort(lx) | ((uint32_t)__bfloat16_as_ushort(ly) << 16);
+}
+
+template <int HD, int NW>
+__global__ void __launch_bounds__(NW * 32)
+attn_mma_kernel(const AttnArgs a) {
+    constexpr int GP = NW * 16;                  // padded query rows
+    constexpr int CH = HD / 8;                   // 16-byte chunks per row
+    constexpr int THREADS = NW * 32;
+    constexpr int TILE_BYTES = TKEYS * HD * 2;
+    extern __shared__ __align__(128) uint8_t sm[];
+    uint8_t* Qh = sm;
+    uint8_t* Ql = Qh + GP * HD * 2;
+    uint8_t* Kt = Ql + GP * HD * 2;              // [2][TKEYS][HD]
+    uint8_t* Vt = Kt + 2 * TILE_BYTES;           // [2][TKEYS][HD]
+    __shared__ int s_last;
+
+    const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = a.n_q / a.n_kv, R = a.R;
+    const int G = g * R;
+    const int qd = a.n_q * HD;
+
+    griddep_wait();
+    griddep_launch_dependents();
+    const int rows = a.seq_rows[b];
+    const int pos0 = a.seq_pos0[b];
+    if (rows == 0) {
+        // sequence not in this step: its rows of the output are zero
+        if (sp == 0) {
+            for (int i = tid; i < G * (HD / 4); i += THREADS) {
+                const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
+                const int m = b * R + rho % R;
+                const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
+                const size_t col = (size_t)(kh * g + rho / R) * HD + d4;
+                *reinterpret_cast<uint2*>(a.out + row * qd + col) = make_uint2(0u, 0u);
+                *reinterpret_cast<uint2*>(a.out + (row + a.TB) * qd + col) = make_uint2(0u, 0u);
+            }
+        }
+        return;
+    }
+    const int total = pos0 + rows;               // keys visible to the last row
+    int chunk = (total + a.splits - 1) / a.splits;
+    chunk = (chunk + TKEYS - 1) / TKEYS * TKEYS;
+    const int k_begin = sp * chunk;
+    const int k_end = min(total, k_begin + chunk);
+    const int n_tiles = k_begin < k_end ? (k_end - k_begin + TKEYS - 1) / TKEYS : 0;
+    const int n_slabs = (G + 15) / 16;
+
+    auto load_tile = [&](int tile, int stage) {
+        const int k0 = k_begin + tile * TKEYS;
+        const uint32_t kdst = smem_u32(Kt + stage * TILE_BYTES), vdst = smem_u32(Vt + stage * TILE_BYTES);
+        for (int i = tid; i < TKEYS * CH; i += THREADS) {
+            const int row = i / CH, c = i % CH;
+            const int key = k0 + row;
+            size_t off = 0;
+            int bytes = 0;
+            if (key < k_end) {
+                const int pslot = key / a.page_size;
+                int page = -1;
+                if (pslot < a.max_pages) page = a.block_table[(size_t)b * a.max_pages + pslot];
+                if (page >= 0 && page < a.n_pages) {       // ids outside the pool read as zeros, never as memory
+                    off = (((size_t)page * a.n_kv + kh) * a.page_size + key % a.page_size) * HD + c * 8;
+                    bytes = 16;
+                }
+            }
+            const uint32_t so = swz<HD>(row, c);
+            cp_async16(kdst + so, a.kp + off, bytes);
+            cp_async16(vdst + so, a.vp + off, bytes);
+        }
+        cp_async_commit();
+    };
+    if (n_tiles > 0) load_tile(0, 0);
+
+    // Q rows of this KV head's group, scaled, as (hi, lo) bf16 in swizzled shared memory
+    for (int i = tid; i < GP * (HD / 4); i += THREADS) {
+        const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
+        const int hl = rho / R, rr = rho % R;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (rho < G && rr < rows) {
+            v = *reinterpret_cast<const float4*>(a.q + (size_t)(b * R + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
+            v.x *= a.scale_log2e; v.y *= a.scale_log2e; v.z *= a.scale_log2e; v.w *= a.scale_log2e;
+        }
+        uint2 h, l;
+        pack_hilo(v.x, v.y, h.x, l.x);
+        pack_hilo(v.z, v.w, h.y, l.y);
+        const uint32_t so = swz<HD>(rho, d4 >> 3) + (uint32_t)((d4 & 7) * 2);
+        *reinterpret_cast<uint2*>(Qh + so) = h;
+        *reinterpret_cast<uint2*>(Ql + so) = l;
+    }
+
+    // per-thread rows of the slab: r0 = lane / 4 and r0 + 8
+    const int rho0 = warp * 16 + (lane >> 2), rho1 = rho0 + 8;
+    const int lim0 = (rho0 < G && rho0 % R < rows) ? min(pos0 + rho0 % R, k_end - 1) : -1;   // last visible key
+    const int lim1 = (rho1 < G && rho1 % R < rows) ? min(pos0 + rho1 % R, k_end - 1) : -1;
+    float o[HD / 8][4];
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const uint32_t qh_base = smem_u32(Qh), ql_base = smem_u32(Ql);
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        const int stage = tile & 1;
+        if (tile + 1 < n_tiles) {
+            load_tile(tile + 1, stage ^ 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        if (warp < n_slabs) {
+            const int k0 = k_begin + tile * TKEYS;
+            const uint32_t kbase = smem_u32(Kt + stage * TILE_BYTES), vbase = smem_u32(Vt + stage * TILE_BYTES);
+            float s[8][4];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
+            const int mi = lane >> 3, li = lane & 7;
+#pragma unroll
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                uint32_t qh[4], ql[4];
+                const uint32_t qo = swz<HD>(warp * 16 + (mi & 1) * 8 + li, ks * 2 + (mi >> 1));
+                ldsm_x4(qh_base + qo, qh);
+                ldsm_x4(ql_base + qo, ql);
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    uint32_t kb[4];
+                    ldsm_x4(kbase + swz<HD>(np * 16 + (mi >> 1) * 8 + li, ks * 2 + (mi & 1)), kb);
+                    mma_bf16(s[2 * np], qh, kb[0], kb[1]);
+                    mma_bf16(s[2 * np], ql, kb[0], kb[1]);
+                    mma_bf16(s[2 * np + 1], qh, kb[2], kb[3]);
+                    mma_bf16(s[2 * np + 1], ql, kb[2], kb[3]);
+                }
+            }
+            // causal / range mask (only tiles that reach past the committed prefix or the split's end)
+            if (k0 + TKEYS > pos0 + 1 || k0 + TKEYS > k_end || lim0 < 0 || lim1 < 0) {
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {
+                    const int key = k0 + nt * 8 + 2 * (lane & 3);
+                    if (key > lim0) s[nt][0] = -INFINITY;
+                    if (key + 1 > lim0) s[nt][1] = -INFINITY;
+                    if (key > lim1) s[nt][2] = -INFINITY;
+                    if (key + 1 > lim1) s[nt][3] = -INFINITY;
+                }
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
+            }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+            const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+            const float al0 = exp2f(m_run[0] - mu0), al1 = exp2f(m_run[1] - mu1);     // 0 while nothing was visible
+            m_run[0] = mn0; m_run[1] = mn1;
+            float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                s[nt][0] = exp2f(s[nt][0] - mu0); s[nt][1] = exp2f(s[nt][1] - mu0);
+                s[nt][2] = exp2f(s[nt][2] - mu1); s[nt][3] = exp2f(s[nt][3] - mu1);
+                ps0 += s[nt][0] + s[nt][1];
+                ps1 += s[nt][2] + s[nt][3];
+            }
+            l_run[0] = l_run[0] * al0 + ps0;
+            l_run[1] = l_run[1] * al1 + ps1;
+#pragma unroll
+            for (int i = 0; i < HD / 8; ++i) { o[i][0] *= al0; o[i][1] *= al0; o[i][2] *= al1; o[i][3] *= al1; }
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) {
+                uint32_t ph[4], pl[4];
+                pack_hilo(s[2 * kb][0], s[2 * kb][1], ph[0], pl[0]);
+                pack_hilo(s[2 * kb][2], s[2 * kb][3], ph[1], pl[1]);
+                pack_hilo(s[2 * kb + 1][0], s[2 * kb + 1][1], ph[2], pl[2]);
+                pack_hilo(s[2 * kb + 1][2], s[2 * kb + 1][3], ph[3], pl[3]);
+#pragma unroll
+                for (int dp = 0; dp < HD / 16; ++dp) {
+                    uint32_t vb[4];
+                    ldsm_x4_trans(vbase + swz<HD>(kb * 16 + (mi & 1) * 8 + li, dp * 2 + (mi >> 1)), vb);
+                    mma_bf16(o[2 * dp], ph, vb[0], vb[1]);
+                    mma_bf16(o[2 * dp], pl, vb[0], vb[1]);
+                    mma_bf16(o[2 * dp + 1], ph, vb[2], vb[3]);
+                    mma_bf16(o[2 * dp + 1], pl, vb[2], vb[3]);
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // this split's partial result
+    const size_t slot = ((size_t)b * a.n_kv + kh) * a.splits + sp;
+    if (warp < n_slabs) {
+        l_run[0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[0], 1);
+        l_run[0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[0], 2);
+        l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], 1);
+        l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], 2);
+        if (n_tiles > 0) {
+            float* op0 = a.o_part + (slot * GP + rho0) * HD + 2 * (lane & 3);
+            float* op1 = a.o_part + (slot * GP + rho1) * HD + 2 * (lane & 3);
+#pragma unroll
+            for (int nt = 0; nt < HD / 8; ++nt) {
+                *reinterpret_cast<float2*>(op0 + nt * 8) = make_float2(o[nt][0], o[nt][1]);
+                *reinterpret_cast<float2*>(op1 + nt * 8) = make_float2(o[nt][2], o[nt][3]);
+            }
+        }
+        if ((lane & 3) == 0) {
+            a.ml_part[slot * GP + rho0] = make_float2(m_run[0], l_run[0]);
+            a.ml_part[slot * GP + rho1] = make_float2(m_run[1], l_run[1]);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int ticket = atomicAdd(&a.counters[b * a.n_kv + kh], 1u);
+        s_last = ticket == (unsigned int)(a.splits - 1);
+        if (s_last) a.counters[b * a.n_kv + kh] = 0u;        // ready for the next layer
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    // merge the splits of this (sequence, KV head) in index order
+    const size_t slot0 = ((size_t)b * a.n_kv + kh) * a.splits;
+    for (int i = tid; i < G * (HD / 4); i += THREADS) {
+        const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
+        const int hl = rho / R, rr = rho % R;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (rr < rows) {
+            float mstar = -INFINITY;
+            for (int s = 0; s < a.splits; ++s) mstar = fmaxf(mstar, __ldcg(&a.ml_part[(slot0 + s) * GP + rho]).x);
+            float den = 0.f;
+            for (int s = 0; s < a.splits; ++s) {
+                const float2 ml = __ldcg(&a.ml_part[(slot0 + s) * GP + rho]);
+                if (ml.x == -INFINITY) continue;
+                const float w = exp2f(ml.x - mstar);
+                den += w * ml.y;
+                const float4 ov = __ldcg(reinterpret_cast<const float4*>(a.o_part + ((slot0 + s) * GP + rho) * HD + d4));
+                acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+            }
+            const float inv = 1.0f / den;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        }
+        const int m = b * R + rr;
+        const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
+        const size_t col = (size_t)(kh * g + hl) * HD + d4;
+        uint2 h, l;
+        pack_hilo(acc.x, acc.y, h.x, l.x);
+        pack_hilo(acc.z, acc.w, h.y, l.y);
+        *reinterpret_cast<uint2*>(a.out + row * qd + col) = h;
+        *reinterpret_cast<uint2*>(a.out + (row + a.TB) * qd + col) = l;
+    }
+}
+
+template <int HD, int NW>
+tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
+    constexpr int GP = NW * 16;
+    const size_t smem = (size_t)2 * GP * HD * 2 + (size_t)4 * TKEYS * HD * 2;
+    static bool done[64] = {false};
+    int dev = 0;
+    TASC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return TASC_EINVAL;
+    if (!done[dev]) {
+        TASC_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<HD, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        done[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)a.splits, (unsigned)a.n_kv, (unsigned)B);
+    cfg.blockDim = dim3(NW * 32, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    ProfScope ps(K_ATT_SPLIT, stream);
+    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_mma_kernel<HD, NW>, a));
+    return TASC_OK;
+}
+
+}  // namespace
+
+int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
+
+size_t attention_mma_scratch_bytes(int B, int n_kv, int hd, int G, int n_splits) {
+    const size_t slots = (size_t)B * n_kv * n_splits * attention_mma_row_pad(G);
+    return slots * hd * sizeof(float) + slots * sizeof(float2);
+}
+
+tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
+                                 const int32_t* block_table, int max_pages, int page_size, long long n_pages,
+                                 const RowPlan& rp, __nv_bfloat16* out, int TB, float* scratch, unsigned int* counters,
+                                 int B, int R, int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream) {
+    const int G = (n_q / n_kv) * R;
+    if (G > 128 || (hd != 32 && hd != 64 && hd != 128)) return TASC_EINVAL;
+    const int GP = attention_mma_row_pad(G);
+    AttnArgs a;
+    a.q = qbuf; a.kp = k_pages; a.vp = v_pages; a.block_table = block_table;
+    a.max_pages = max_pages; a.page_size = page_size; a.n_pages = n_pages;
+    a.seq_pos0 = rp.seq_pos0; a.seq_rows = rp.seq_rows;
+    a.out = out; a.TB = TB;
+    const size_t slots = (size_t)B * n_kv * n_splits * GP;
+    a.o_part = scratch;
+    a.ml_part = reinterpret_cast<float2*>(scratch + slots * hd);
+    a.counters = counters;
+    a.R = R; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits;
+    a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
+    if (GP == 64) {
+        if (hd == 32) return launch_inst<32, 4>(a, B, stream);
+        if (hd == 64) return launch_inst<64, 4>(a, B, stream);
+        return launch_inst<128, 4>(a, B, stream);
+    }
+    if (hd == 32) return launch_inst<32, 8>(a, B, stream);
+    if (hd == 64) return launch_inst<64, 8>(a, B, stream);
+    return launch_inst<128, 8>(a, B, stream);
+}
+
+}  // namespace tasc

@@ -9,10 +9,19 @@
 
 #include "tasc.h"
 
+namespace tasc {
+// Remembers the most recent failing CUDA call (what, where) for tasc_last_error(); defined in profile.cu.
+void note_cuda_error(cudaError_t e, const char* expr, const char* file, int line);
+}
+
 #define TASC_CUDA_TRY(expr)                                   \
     do {                                                      \
         cudaError_t e__ = (expr);                             \
-        if (e__ != cudaSuccess) { (void)cudaGetLastError(); return TASC_ECUDA; } \
+        if (e__ != cudaSuccess) {                             \
+            ::tasc::note_cuda_error(e__, #expr, __FILE__, __LINE__); \
+            (void)cudaGetLastError();                         \
+            return TASC_ECUDA;                                \
+        }                                                     \
     } while (0)
 
 namespace tasc {
@@ -116,6 +125,49 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long lo
         if (clock64() - t0 > budget) return false;
     }
     return true;
+}
+
+// ---------------------------------------------------------------- thread-block clusters, distributed shared memory
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of every CTA of the cluster must execute both halves, warp-convergently.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// Address of this CTA's shared-memory location `addr` in the CTA of rank `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// ---------------------------------------------------------------- programmatic dependent launch
+// wait: returns once every grid this one depends on has completed and its writes are visible (no-op for a
+// normal launch).  launch_dependents: lets the next grid in the stream start its prologue.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Adds to the barrier's pending transaction bytes without arriving.
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// (hi, lo) split of a float32: hi = bf16(v), lo = bf16(v - hi).
+__device__ __forceinline__ void split_bf16(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
 // ---------------------------------------------------------------- TMA (tiled bulk tensor load, no multicast)

@@ -1,0 +1,464 @@
+// Projection GEMMs of the verify forward with their consumers fused in: tcgen05 MMA with float32
+// accumulators in TMEM, weights streamed by TMA, split-K reduced through distributed shared memory
+// inside a thread-block cluster, and the stage that follows the product (RoPE + KV append, residual +
+// next norm's input, SiLU * up, LM-head argmax) done on the reduced tile before anything goes to HBM.
+//
+// Shape of the work.  Y^T[128 features][tokens] = W[128 rows][K] * X^T, operands swapped because the
+// step has few token rows (M = B * (k+1)) and large weight matrices: the weight tile supplies UMMA M,
+// the token rows UMMA N.  Activations are float32 values carried as (hi, lo) bf16 row pairs in the
+// tile-local layout [TB hi rows][TB lo rows], both halves go through one MMA (N = 2 TB) and the
+// accumulator columns j and j + TB are added afterwards.
+//
+// Split-K.  The narrow matrices of small models give few 128-row tiles, so a cluster of S CTAs shares
+// one output tile and splits the k-range.  Each CTA copies its accumulator to its own shared memory;
+// after a cluster barrier CTA r sums, in fixed rank order, the S copies of its 1/S share of the token
+// columns (ld.shared::cluster) and runs the epilogue for them.  No partial sum reaches global memory,
+// no atomics, and the result does not depend on timing.
+//
+// RMSNorm without a row-wide pass.  The producer of a normalised input writes x * gain (as hi/lo)
+// and, per 128-feature tile, the row's partial sum of squares; the consumer GEMM multiplies its
+// output row by 1 / sqrt(mean(x^2) + eps), which commutes with the product.
+//
+// Launch overlap.  Kernels are launched with programmatic stream serialisation: a CTA sets up its
+// barriers and TMEM and streams the first weight tiles of its k-range into the ring (weights do not
+// depend on earlier kernels), then waits for the preceding grid (griddepcontrol.wait) before it
+// touches activations, and releases the next grid once its last weight load has been issued.
+//
+// Warp roles (192 threads): warps 0-3 epilogue (TMEM lane quarter w), warp 4 TMA producer, warp 5
+// TMEM allocation + MMA issue.  Every mbarrier wait is bounded; a wait that runs out records
+// TASC_ETIMEOUT, the CTA still takes part in the cluster barriers, frees its TMEM and returns.
+#include "kernels.h"
+
+#include <algorithm>
+
+namespace tasc {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int UMMA_K = 16;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int THREADS = 192;
+constexpr int LM_SMEM = 4 * 256 * 8;
+constexpr int MAX_DYN_SMEM = 226 * 1024;      // 227 KB per CTA minus the kernel's static shared memory
+
+__device__ __forceinline__ float4 shfl_xor4(float4 v, int d) {
+    float4 r;
+    r.x = __shfl_xor_sync(0xFFFFFFFFu, v.x, d);
+    r.y = __shfl_xor_sync(0xFFFFFFFFu, v.y, d);
+    r.z = __shfl_xor_sync(0xFFFFFFFFu, v.z, d);
+    r.w = __shfl_xor_sync(0xFFFFFFFFu, v.w, d);
+    return r;
+}
+
+// Four consecutive values -> (hi, lo) bf16 quadruples, 8 bytes each.
+__device__ __forceinline__ void store_hilo4(__nv_bfloat16* hi_ptr, __nv_bfloat16* lo_ptr, const float v[4]) {
+    __nv_bfloat16 h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) split_bf16(v[e], h[e], l[e]);
+    uint2 ph, pl;
+    ph.x = (uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16);
+    ph.y = (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16);
+    pl.x = (uint32_t)__bfloat16_as_ushort(l[0]) | ((uint32_t)__bfloat16_as_ushort(l[1]) << 16);
+    pl.y = (uint32_t)__bfloat16_as_ushort(l[2]) | ((uint32_t)__bfloat16_as_ushort(l[3]) << 16);
+    *reinterpret_cast<uint2*>(hi_ptr) = ph;
+    *reinterpret_cast<uint2*>(lo_ptr) = pl;
+}
+__device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, const float v[4]) {
+    uint2 u;
+    u.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[0])) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[1])) << 16);
+    u.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[2])) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[3])) << 16);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const FusedArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+
+    const int BN = a.BN, stages = a.stages, TB = a.TB;
+    const uint32_t b_stage_bytes = (uint32_t)BN * BK * 2;
+    const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.data_bytes);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8u * stages;
+    const uint32_t bar_acc = bar_full + 16u * stages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * stages + 1);
+    float* s_inv = reinterpret_cast<float*>(bars + 2 * stages + 2);                       // [128]
+    unsigned long long* s_arg = reinterpret_cast<unsigned long long*>(s_inv + 128);       // [4][256], LM head only
+    float* red = reinterpret_cast<float*>(smem);                                          // [TB][128], reuses the ring
+
+    const int S = (int)cluster_nctarank();
+    const int rank = (int)cluster_ctarank();
+    const int out_tile = blockIdx.y, m_tile = blockIdx.z;
+    const int kb_begin = (int)(((long long)a.num_kb * rank) / S);
+    const int kb_end = (int)(((long long)a.num_kb * (rank + 1)) / S);
+    const int n_kb = kb_end - kb_begin;
+    const int f0 = out_tile * (EPI == EPI_SWIGLU ? 64 : BM);   // first output feature of the tile
+    const int m0 = m_tile * BN;                                // first row of the tile in the activation buffer
+    const int t0 = m_tile * TB;                                // first token of the tile
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t ncols = 32;
+    while ((int)ncols < BN) ncols <<= 1;
+    __shared__ int s_fail;              // a bounded wait ran out somewhere in this CTA
+    auto fail = [&]() { set_status(a.status, TASC_ETIMEOUT); s_fail = 1; };
+
+    if (threadIdx.x == 0) {
+        s_fail = 0;
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(bar_full + 8u * s, 1);
+            mbar_init(bar_empty + 8u * s, 1);
+        }
+        mbar_init(bar_acc, 1);
+        fence_barrier_init();
+    }
+    if (warp == 4 && lane == 0) {
+        tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmX);
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(tmem_slot), ncols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first();   // weights are read once per step
+            const uint64_t pol_x = policy_evict_last();    // token rows are re-read by every CTA
+            auto load_w = [&](int i, uint32_t dstA, uint32_t bar) {
+                const int kc = (kb_begin + i) * BK;
+                if (EPI == EPI_SWIGLU) {                   // 64 gate rows, then the 64 matching up rows
+                    tma_load_2d_hint(dstA, &tmW, kc, f0, bar, pol_w);
+                    tma_load_2d_hint(dstA + A_STAGE_BYTES / 2, &tmW, kc, a.N + f0, bar, pol_w);
+                } else {
+                    tma_load_2d_hint(dstA, &tmW, kc, f0, bar, pol_w);
+                }
+            };
+            // weights of the first stages do not depend on the preceding grid: start them now
+            const int pre = n_kb < stages ? n_kb : stages;
+            for (int i = 0; i < pre; ++i) {
+                const uint32_t dstA = smem_u32(smem + (size_t)i * stage_bytes);
+                mbar_expect_tx_only(bar_full + 8u * i, A_STAGE_BYTES);
+                load_w(i, dstA, bar_full + 8u * i);
+            }
+            griddep_wait();
+            for (int i = 0; i < pre; ++i) {
+                const uint32_t dstB = smem_u32(smem + (size_t)i * stage_bytes) + A_STAGE_BYTES;
+                mbar_expect_tx(bar_full + 8u * i, b_stage_bytes);
+                tma_load_2d_hint(dstB, &tmX, (kb_begin + i) * BK, m0, bar_full + 8u * i, pol_x);
+            }
+            for (int i = pre; i < n_kb; ++i) {
+                const int s = i % stages;
+                const uint32_t round = (uint32_t)(i / stages);
+                if (!mbar_wait(bar_empty + 8u * s, (round & 1u) ^ 1u)) { fail(); break; }
+                const uint32_t dstA = smem_u32(smem + (size_t)s * stage_bytes);
+                mbar_expect_tx(bar_full + 8u * s, stage_bytes);
+                load_w(i, dstA, bar_full + 8u * s);
+                tma_load_2d_hint(dstA + A_STAGE_BYTES, &tmX, (kb_begin + i) * BK, m0, bar_full + 8u * s, pol_x);
+            }
+            griddep_launch_dependents();
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+            bool ok = true;
+            for (int i = 0; i < n_kb && ok; ++i) {
+                const int s = i % stages;
+                const uint32_t round = (uint32_t)(i / stages);
+                if (!mbar_wait(bar_full + 8u * s, round & 1u)) { fail(); ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                    const uint64_t da = umma_desc_k_sw128(sa + kk * UMMA_K * 2);
+                    const uint64_t db = umma_desc_k_sw128(sb + kk * UMMA_K * 2);
+                    umma_bf16(tmem_base, da, db, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(bar_empty + 8u * s);
+            }
+            if (ok) umma_commit(bar_acc);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue, part 1: accumulator -> shared memory
+        griddep_wait();
+        if (EPI == EPI_QKV || EPI == EPI_SWIGLU || EPI == EPI_LM || (EPI == EPI_PLAIN && a.ssq_in)) {
+            for (int t = threadIdx.x; t < TB; t += 128) {
+                const int m = t0 + t;
+                float ss = 0.f;
+                if (m < a.M)
+                    for (int j = 0; j < a.ssq_slots; ++j) ss += a.ssq_in[(size_t)m * a.ssq_slots + j];
+                s_inv[t] = 1.0f / sqrtf(ss * a.inv_d + a.eps);
+            }
+        }
+        bool have = n_kb > 0;
+        if (have && !mbar_wait(bar_acc, 0)) { fail(); have = false; }
+        tc_fence_after();
+        asm volatile("bar.sync 1, 128;" ::: "memory");          // s_inv visible to the four epilogue warps
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        for (int c = 0; c < TB / 16; ++c) {
+            uint32_t r[16];
+            if (have) {
+                tmem_ld16(lane_base + (uint32_t)(c * 16), r);
+                if (a.pair) {
+                    uint32_t r2[16];
+                    tmem_ld16(lane_base + (uint32_t)(TB + c * 16), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                } else {
+                    tmem_ld_wait();
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) r[j] = 0u;
+            }
+            if (EPI == EPI_LM) {
+                const int f = f0 + warp * 32 + lane;
+                const bool f_ok = f < a.N;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int n = c * 16 + j;
+                    const float v = __uint_as_float(r[j]);
+                    const uint32_t key = f_ok ? float_key(v) : 0u;
+                    const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
+                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
+                    if (lane == 0) {
+                        const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
+                        s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
+                    }
+                    if (a.logits && f_ok && t0 + n < a.M) a.logits[(size_t)(t0 + n) * a.N + f] = v * s_inv[n];
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) red[(c * 16 + j) * BM + warp * 32 + lane] = __uint_as_float(r[j]);
+            }
+        }
+        if (EPI == EPI_LM) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            for (int n = threadIdx.x; n < TB; n += 128) {
+                if (t0 + n < a.M) {
+                    unsigned long long best = s_arg[n];
+                    best = max(best, s_arg[256 + n]);
+                    best = max(best, s_arg[512 + n]);
+                    best = max(best, s_arg[768 + n]);
+                    atomicMax(&a.argmax[t0 + n], best);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    cluster_arrive();
+    cluster_wait();
+
+    if (warp < 4 && EPI != EPI_LM) {
+        // ------------------------------------------------------------ epilogue, part 2: this CTA's share of the token columns
+        int valid = a.M - t0;
+        valid = valid > TB ? TB : valid;
+        const int per = (valid + S - 1) / S;
+        const int c0 = rank * per;
+        const int c1 = c0 + per < valid ? c0 + per : valid;
+        const uint32_t red_addr = smem_u32(red);
+        for (int t = c0 + warp; t < c1; t += 4) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            const uint32_t off = red_addr + (uint32_t)((t * BM + 4 * lane) * 4);
+            for (int s = 0; s < S; ++s) {
+                const float4 p = ld_cluster_f4(cluster_map(off, (uint32_t)s));
+                acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+            }
+            const int m = t0 + t;
+            if (EPI == EPI_PLAIN) {
+                const float sc = a.ssq_in ? s_inv[t] : 1.0f;
+                const float v[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int f = f0 + 4 * lane + e;
+                    if (f < a.N) a.y[(size_t)m * a.N + f] = v[e];
+                }
+            } else if (EPI == EPI_QKV) {
+                const float sc = s_inv[t];
+                acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
+                const int hd = a.hd, half = hd >> 1;
+                const float4 partner = shfl_xor4(acc, half >> 2);
+                const int f = f0 + 4 * lane;
+                const int qd = a.n_q * hd, kvd = a.n_kv * hd;
+                int pos = a.row_pos[m];
+                if (pos >= a.max_positions) { set_status(a.status, TASC_EINVAL); pos = -1; }
+                float v[4] = {acc.x, acc.y, acc.z, acc.w};
+                if (f < qd + kvd && pos >= 0) {
+                    const int i = f % hd;
+                    const float4* cs = reinterpret_cast<const float4*>(a.rope + (size_t)pos * half + (i % half));
+                    const float4 cs01 = cs[0], cs23 = cs[1];        // (cos, sin) of four consecutive pair indices
+                    const float co[4] = {cs01.x, cs01.z, cs23.x, cs23.z};
+                    const float si[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
+                    const float pv[4] = {partner.x, partner.y, partner.z, partner.w};
+                    const float sgn = i < half ? -1.0f : 1.0f;      // first half: a c - b s; second half: b c + a s
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) v[e] = v[e] * co[e] + sgn * pv[e] * si[e];
+                }
+                if (f < qd) {
+                    if (pos < 0) { v[0] = v[1] = v[2] = v[3] = 0.f; }
+                    *reinterpret_cast<float4*>(a.qbuf + (size_t)m * qd + f) = make_float4(v[0], v[1], v[2], v[3]);
+                } else if (f < qd + 2 * kvd && pos >= 0) {
+                    const int b = m / a.R;
+                    const int pslot = pos / a.page_size;
+                    int page = -1;
+                    if (pslot < a.max_pages) page = a.block_table[(size_t)b * a.max_pages + pslot];
+                    if (page < 0 || page >= a.n_pages) {
+                        set_status(a.status, TASC_ENOKV);
+                    } else {
+                        const bool is_k = f < qd + kvd;
+                        const int g = f - qd - (is_k ? 0 : kvd);
+                        const int kh = g / hd, i = g % hd;
+                        __nv_bfloat16* base = is_k ? a.k_pages : a.v_pages;
+                        store_bf16x4(base + (((size_t)page * a.n_kv + kh) * a.page_size + pos % a.page_size) * hd + i, v);
+                    }
+                }
+            } else if (EPI == EPI_RESID) {
+                const int f = f0 + 4 * lane;
+                float ss = 0.f;
+                if (f < a.N) {
+                    float4* xp = reinterpret_cast<float4*>(a.x + (size_t)m * a.N + f);
+                    float4 xv = *xp;
+                    xv.x += acc.x; xv.y += acc.y; xv.z += acc.z; xv.w += acc.w;
+                    *xp = xv;
+                    ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
+                    const float4 g = *reinterpret_cast<const float4*>(a.gain + f);
+                    const float v[4] = {xv.x * g.x, xv.y * g.y, xv.z * g.z, xv.w * g.w};
+                    const size_t row = (size_t)(m / TB) * (2 * TB) + (m % TB);
+                    store_hilo4(a.a_out + row * a.N + f, a.a_out + (row + TB) * a.N + f, v);
+                }
+                ss = warp_sum(ss);
+                if (lane == 0) a.ssq_out[(size_t)m * a.ssq_out_slots + out_tile] = ss;
+            } else if (EPI == EPI_SWIGLU) {
+                const float sc = s_inv[t];
+                const float4 up = shfl_xor4(acc, 16);              // lanes 0-15 hold gate features, 16-31 the up features
+                const int j = f0 + 4 * lane;
+                if (lane < 16 && j < a.N) {
+                    const float g[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
+                    const float u[4] = {up.x * sc, up.y * sc, up.z * sc, up.w * sc};
+                    float v[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) v[e] = g[e] / (1.0f + expf(-g[e])) * u[e];
+                    const size_t row = (size_t)(m / TB) * (2 * TB) + (m % TB);
+                    store_hilo4(a.a_out + row * a.N + j, a.a_out + (row + TB) * a.N + j, v);
+                }
+            }
+        }
+    }
+    // peers may still be reading this CTA's shared memory
+    cluster_arrive();
+    cluster_wait();
+    if (s_fail && warp == 4 && lane == 0) {
+        // after a timeout: give this CTA's own tile loads that may still be in flight a bounded time to land
+        for (int i = 0; i < n_kb; ++i) {
+            const int s = i % stages;
+            if (i + stages >= n_kb) (void)mbar_wait(bar_full + 8u * s, (uint32_t)(i / stages) & 1u, 2000000ll);
+        }
+    }
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, ncols);
+    }
+}
+
+template <int EPI>
+tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const FusedArgs& a, const FusedPlan& p, int kind,
+                       cudaStream_t stream) {
+    static bool attr_done[64] = {false};
+    int dev = 0;
+    TASC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return TASC_EINVAL;
+    if (!attr_done[dev]) {
+        TASC_CUDA_TRY(cudaFuncSetAttribute(gemm_fused_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM));
+        attr_done[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.S, (unsigned)p.out_tiles, (unsigned)p.m_tiles);
+    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[2];
+    int n = 0;
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (p.S > 1) {
+        at[n].id = cudaLaunchAttributeClusterDimension;
+        at[n].val.clusterDim.x = (unsigned)p.S;
+        at[n].val.clusterDim.y = 1;
+        at[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = at;
+    cfg.numAttrs = n;
+    ProfScope ps(kind, stream);
+    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_fused_kernel<EPI>, *tmW, *tmX, a));
+    return TASC_OK;
+}
+
+}  // namespace
+
+FusedPlan plan_fused(int M, int N, int K, int epi) {
+    FusedPlan p;
+    p.TB = gemm_token_tile(M, true);
+    p.BN = 2 * p.TB;
+    p.m_tiles = (M + p.TB - 1) / p.TB;
+    p.out_tiles = epi == EPI_SWIGLU ? (N + 63) / 64 : (N + BM - 1) / BM;
+    p.num_kb = (K + BK - 1) / BK;
+    const int tiles = p.out_tiles * p.m_tiles;
+    int S = 1;
+    if (epi != EPI_LM) {
+        S = std::max(1, 148 / tiles);
+        S = std::min(S, 8);
+        S = std::min(S, p.num_kb);
+    }
+    p.S = S;
+    const int kb_per = (p.num_kb + S - 1) / S;
+    const int stage_bytes = A_STAGE_BYTES + p.BN * BK * 2;
+    int ncols = 32;
+    while (ncols < p.BN) ncols <<= 1;
+    // Up to 128 accumulator columns: about 100 KB so that two CTAs (or this grid and the next one's
+    // prologue) share an SM; wider tiles take one CTA per SM and a deeper ring.
+    const int budget = ncols <= 128 ? 96 * 1024 : 192 * 1024;
+    int st = budget / stage_bytes;
+    st = std::max(2, std::min(st, 8));
+    st = std::min(st, std::max(2, kb_per));
+    p.stages = st;
+    p.data_bytes = std::max(st * stage_bytes, p.TB * BM * 4);
+    int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4 + (epi == EPI_LM ? LM_SMEM : 0);
+    // TMEM columns held by co-resident CTAs must never exceed 512, or CTAs of different clusters can
+    // block each other's allocation while waiting at a cluster barrier: shared memory limits residency.
+    smem = std::max(smem, ncols * 454 + 1);
+    p.smem_bytes = std::min(smem, MAX_DYN_SMEM);
+    return p;
+}
+
+tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
+                              cudaStream_t stream) {
+    if (a.M <= 0 || a.N <= 0 || a.K <= 0) return TASC_EINVAL;
+    a.num_kb = p.num_kb; a.BN = p.BN; a.TB = p.TB; a.stages = p.stages; a.pair = 1; a.data_bytes = p.data_bytes;
+    switch (epi) {
+        case EPI_PLAIN:  return launch_epi<EPI_PLAIN>(tmW, tmX, a, p, K_GEMM, stream);
+        case EPI_QKV:    return launch_epi<EPI_QKV>(tmW, tmX, a, p, K_GEMM, stream);
+        case EPI_RESID:  return launch_epi<EPI_RESID>(tmW, tmX, a, p, K_GEMM, stream);
+        case EPI_SWIGLU: return launch_epi<EPI_SWIGLU>(tmW, tmX, a, p, K_GEMM, stream);
+        case EPI_LM:     return launch_epi<EPI_LM>(tmW, tmX, a, p, K_GEMM_LM, stream);
+        default: return TASC_EINVAL;
+    }
+}
+
+}  // namespace tasc

@@ -43,6 +43,49 @@ tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, flo
                              cudaStream_t stream);
 tasc_status gemm_set_attributes();
 
+// ------------------------------------------------------------------ fused projection GEMMs (gemm_fused.cu)
+// What happens to the reduced output tile before anything is written to global memory.
+enum Epi {
+    EPI_PLAIN,    // y[m][f] = acc (times the row's RMS factor when ssq_in is given)
+    EPI_QKV,      // acc * rms factor; RoPE on q and k heads; q -> qbuf, k and v -> KV pages
+    EPI_RESID,    // x[m][f] += acc; a_out = (hi, lo) of x * gain; ssq_out[m][tile] = sum over the tile of x^2
+    EPI_SWIGLU,   // tile = 64 gate rows + the 64 matching up rows; a_out = (hi, lo) of SiLU(gate) * up, both times the rms factor
+    EPI_LM        // per token row an atomic max of (value, id) in argmax[m]; logits (nullable) get the scaled rows
+};
+struct FusedArgs {
+    int M, N, K;                       // token rows, output features (EPI_SWIGLU: d_ff), reduction length
+    int num_kb, BN, TB, stages, pair, data_bytes;      // filled in by launch_gemm_fused from the plan
+    const float* ssq_in;               // [M][ssq_slots] partial sums of squares of the input rows (null: no scaling)
+    int ssq_slots;
+    float inv_d, eps;                  // rms factor = 1 / sqrt(sum(ssq) * inv_d + eps)
+    float* y;                          // EPI_PLAIN
+    const int* row_pos;                // EPI_QKV: position of each row, -1 = unused
+    const float2* rope;
+    float* qbuf;
+    __nv_bfloat16 *k_pages, *v_pages;
+    const int32_t* block_table;
+    int max_pages, page_size;
+    long long n_pages;
+    int R, n_q, n_kv, hd, max_positions;
+    float* x;                          // EPI_RESID
+    const float* gain;
+    float* ssq_out;
+    int ssq_out_slots;
+    __nv_bfloat16* a_out;              // EPI_RESID / EPI_SWIGLU: activation buffer of the next GEMM, [tiles][2 TB][N]
+    unsigned long long* argmax;        // EPI_LM
+    float* logits;
+    int* status;
+};
+struct FusedPlan {
+    int TB, BN, m_tiles, out_tiles, num_kb;
+    int S;             // cluster size = k-splits
+    int stages, data_bytes, smem_bytes;
+};
+FusedPlan plan_fused(int M, int N, int K, int epi);
+// tmW: weight map with box rows 128 (64 for EPI_SWIGLU); tmX: (hi, lo) activation map with box rows 2 TB.
+tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
+                              cudaStream_t stream);
+
 // ------------------------------------------------------------------ float32 GEMM for the f32 model (gemm_simt.cu)
 // Same contract with splits = 1: P[0][m][n].
 void launch_gemm_f32(const float* X, const float* W, float* partials, int M, int N, int K,
@@ -58,10 +101,15 @@ struct RowPlan {              // per-step row bookkeeping, all device pointers i
 // Rows of a verify step: [last committed token, drafts] at positions len-1 ..; skipped when len >= stop_len.
 void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len,
                         const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
-                        cudaStream_t stream);
+                        unsigned int* counters, int n_counters, cudaStream_t stream);
 // Rows of prefill chunk c: committed tokens c*R .. c*R+R-1, limited to positions <= len-2.
 void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
-                         int chunk, int vocab, int* status, cudaStream_t stream);
+                         int chunk, int vocab, int* status, unsigned int* counters, int n_counters, cudaStream_t stream);
+// (both also zero `counters`, the attention merge tickets, when given)
+
+// bf16 model: x[m] = embed[tok]; a_out = (hi, lo) of x * gain; ssq[m][0] = sum x^2, other slots 0; argmax[m] = 0.
+void launch_embed_scaled(const __nv_bfloat16* embed, const int* row_tok, const float* gain, float* x, __nv_bfloat16* a_out,
+                         float* ssq, int ssq_slots, unsigned long long* argmax, int M, int d, int TB, cudaStream_t stream);
 
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
@@ -106,5 +154,14 @@ void launch_attention(const float* qbuf, const T* k_pages, const T* v_pages, con
                       int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream);
 size_t attention_scratch_bytes(int B, int R, int n_q, int hd, int n_splits);
 int attention_splits(int B, int n_kv, int max_ctx);
+
+
+// ------------------------------------------------------------------ tensor-core attention for bf16 models (attention_mma.cu)
+// Same contract as launch_attention; the result goes to `out` as (hi, lo) bf16 rows.  counters: B * n_kv zeroed words.
+tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
+                                 const int32_t* block_table, int max_pages, int page_size, long long n_pages,
+                                 const RowPlan& rp, __nv_bfloat16* out, int TB, float* scratch, unsigned int* counters,
+                                 int B, int R, int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream);
+size_t attention_mma_scratch_bytes(int B, int n_kv, int hd, int G, int n_splits);
 
 }  // namespace tasc

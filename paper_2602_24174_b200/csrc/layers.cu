@@ -19,8 +19,10 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 __global__ void rows_verify_kernel(RowPlan rp, const int32_t* tokens, int64_t stride, const int32_t* len,
-                                   const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status) {
+                                   const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
+                                   unsigned int* counters, int n_counters) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int c = i; c < n_counters; c += gridDim.x * blockDim.x) counters[c] = 0u;
     if (i >= B * R) return;
     const int b = i / R, r = i % R;
     const int L = len[b];
@@ -40,8 +42,9 @@ __global__ void rows_verify_kernel(RowPlan rp, const int32_t* tokens, int64_t st
 }
 
 __global__ void rows_prefill_kernel(RowPlan rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
-                                    int chunk, int vocab, int* status) {
+                                    int chunk, int vocab, int* status, unsigned int* counters, int n_counters) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int c = i; c < n_counters; c += gridDim.x * blockDim.x) counters[c] = 0u;
     if (i >= B * R) return;
     const int b = i / R, r = i % R;
     const int L = len[b];
@@ -80,6 +83,26 @@ embed_norm_kernel(const T* __restrict__ embed, const int* __restrict__ row_tok, 
     const float inv = 1.0f / sqrtf(block_sum(ss, red) / (float)d + eps);
     for (int j = threadIdx.x; j < d; j += blockDim.x)
         ActStore<T>::put(h, m, j, d, TB, x[(size_t)m * d + j] * inv * gain[j]);
+}
+
+// bf16 model: the RMS factor is applied by the consumer GEMM, so the row leaves here as x * gain plus its sum of squares
+__global__ void __launch_bounds__(128)
+embed_scaled_kernel(const __nv_bfloat16* __restrict__ embed, const int* __restrict__ row_tok, const float* __restrict__ gain,
+                    float* __restrict__ x, __nv_bfloat16* __restrict__ a_out, float* __restrict__ ssq, int ssq_slots,
+                    unsigned long long* argmax, int d, int TB) {
+    __shared__ float red[4];
+    const int m = blockIdx.x;
+    const __nv_bfloat16* e = embed + (size_t)row_tok[m] * d;
+    float ss = 0.f;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float v = __bfloat162float(e[j]);
+        x[(size_t)m * d + j] = v;
+        ss += v * v;
+        ActStore<__nv_bfloat16>::put(a_out, m, j, d, TB, v * gain[j]);
+    }
+    ss = block_sum(ss, red);
+    for (int j = threadIdx.x; j < ssq_slots; j += blockDim.x) ssq[(size_t)m * ssq_slots + j] = j == 0 ? ss : 0.f;
+    if (threadIdx.x == 0 && argmax) argmax[m] = 0ull;
 }
 
 // x[m] += sum_s P[s][m]; h[m] = RMSNorm(x[m]) * gain
@@ -270,20 +293,27 @@ __global__ void min_generated_kernel(const int32_t* len, const int32_t* prompt_l
 
 void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len,
                         const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
-                        cudaStream_t stream) {
+                        unsigned int* counters, int n_counters, cudaStream_t stream) {
     ProfScope ps(K_ROWS, stream);
-    rows_verify_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, stop_len, drafts, B, R, vocab, status);
+    rows_verify_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, stop_len, drafts, B, R, vocab, status,
+                                                                counters, n_counters);
 }
 void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
-                         int chunk, int vocab, int* status, cudaStream_t stream) {
+                         int chunk, int vocab, int* status, unsigned int* counters, int n_counters, cudaStream_t stream) {
     ProfScope ps(K_ROWS, stream);
-    rows_prefill_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, B, R, chunk, vocab, status);
+    rows_prefill_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, B, R, chunk, vocab, status,
+                                                                 counters, n_counters);
 }
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
                        int TB, cudaStream_t stream) {
     ProfScope ps(K_EMBED, stream);
     embed_norm_kernel<T><<<M, 128, 0, stream>>>(embed, row_tok, gain, eps, x, h, d, TB);
+}
+void launch_embed_scaled(const __nv_bfloat16* embed, const int* row_tok, const float* gain, float* x, __nv_bfloat16* a_out,
+                         float* ssq, int ssq_slots, unsigned long long* argmax, int M, int d, int TB, cudaStream_t stream) {
+    ProfScope ps(K_EMBED, stream);
+    embed_scaled_kernel<<<M, 128, 0, stream>>>(embed, row_tok, gain, x, a_out, ssq, ssq_slots, argmax, d, TB);
 }
 template <typename T>
 void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,

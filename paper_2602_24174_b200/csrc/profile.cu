@@ -3,6 +3,7 @@
 #include "kernels.h"
 
 #include <atomic>
+#include <cstdio>
 #include <mutex>
 #include <vector>
 
@@ -33,7 +34,17 @@ cudaEvent_t get_event() {
     return e;
 }
 
+char g_last_error[512] = "";
+
 }  // namespace
+
+void note_cuda_error(cudaError_t e, const char* expr, const char* file, int line) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    const char* base = file;
+    for (const char* c = file; *c; ++c)
+        if (*c == '/') base = c + 1;
+    snprintf(g_last_error, sizeof(g_last_error), "%s (%s) at %s:%d in `%s`", cudaGetErrorName(e), cudaGetErrorString(e), base, line, expr);
+}
 
 void prof_begin(int kind, cudaStream_t s) {
     g_launches[kind].fetch_add(1, std::memory_order_relaxed);
@@ -85,6 +96,8 @@ extern "C" tasc_status tasc_profile_read(double* ms_by_kind, int64_t* timed_laun
     g_spans.clear();
     return TASC_OK;
 }
+
+extern "C" const char* tasc_last_error(void) { return g_last_error; }
 
 extern "C" tasc_status tasc_launch_counts(int64_t* launches_by_kind, int32_t n) {
     if (!launches_by_kind || n < K_COUNT) return TASC_EINVAL;
