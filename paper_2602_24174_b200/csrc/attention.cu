@@ -182,11 +182,13 @@ size_t att_smem_bytes(int G, int hd) {
 
 }  // namespace
 
+// Key-range splits per (sequence, KV head): enough CTAs to cover the SMs about twice, at least two
+// 64-key tiles per split, at most 16 (the merge reads every split).
 int attention_splits(int B, int n_kv, int max_ctx) {
     int s = (296 + B * n_kv - 1) / (B * n_kv);
-    const int by_len = (max_ctx + 63) / 64;
+    const int by_len = (max_ctx + 127) / 128;
     if (s > by_len) s = by_len;
-    if (s > 64) s = 64;
+    if (s > 16) s = 16;
     return s < 1 ? 1 : s;
 }
 

@@ -4,7 +4,7 @@
 // The kernel is bound by streaming K and V from HBM once; the tensor cores only have to keep up with
 // that stream, which a float32 SIMT formulation cannot do beyond a few sequences.  A CTA owns one
 // (sequence, KV head, key range): the key range of a sequence is split over several CTAs because the
-// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a two-stage cp.async pipeline
+// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a 3-4 stage cp.async pipeline
 // (16-byte vectors, every page of a KV head is one contiguous run) into XOR-swizzled shared memory;
 // warp w computes the 16-row slab w of S = Q K^T and O += P V with mma.sync m16n8k16 (ldmatrix
 // fragments, V through ldmatrix.trans) and keeps an online softmax per row in registers.
@@ -80,6 +80,9 @@ __device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32
     lo = (uint32_t)__bfloat16_as_ushort(lx) | ((uint32_t)__bfloat16_as_ushort(ly) << 16);
 }
 
+// ring depth of the K/V tile pipeline: enough bytes in flight per CTA to cover the memory latency
+template <int HD> struct Ring { static constexpr int STAGES = HD >= 128 ? 3 : 4; };
+
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32)
 attn_mma_kernel(const AttnArgs a) {
@@ -87,11 +90,12 @@ attn_mma_kernel(const AttnArgs a) {
     constexpr int CH = HD / 8;                   // 16-byte chunks per row
     constexpr int THREADS = NW * 32;
     constexpr int TILE_BYTES = TKEYS * HD * 2;
+    constexpr int STAGES = Ring<HD>::STAGES;
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t* Qh = sm;
     uint8_t* Ql = Qh + GP * HD * 2;
-    uint8_t* Kt = Ql + GP * HD * 2;              // [2][TKEYS][HD]
-    uint8_t* Vt = Kt + 2 * TILE_BYTES;           // [2][TKEYS][HD]
+    uint8_t* Kt = Ql + GP * HD * 2;              // [STAGES][TKEYS][HD]
+    uint8_t* Vt = Kt + STAGES * TILE_BYTES;      // [STAGES][TKEYS][HD]
     __shared__ int s_last;
 
     const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
@@ -100,11 +104,13 @@ attn_mma_kernel(const AttnArgs a) {
     const int G = g * R;
     const int qd = a.n_q * HD;
 
-    griddep_wait();
-    griddep_launch_dependents();
+    // The row plan, the block table and the K/V of committed positions were written before the
+    // preceding grid started, so they may be read ahead of griddepcontrol.wait.
     const int rows = a.seq_rows[b];
     const int pos0 = a.seq_pos0[b];
     if (rows == 0) {
+        griddep_wait();
+        griddep_launch_dependents();
         // sequence not in this step: its rows of the output are zero
         if (sp == 0) {
             for (int i = tid; i < G * (HD / 4); i += THREADS) {
@@ -147,9 +153,21 @@ attn_mma_kernel(const AttnArgs a) {
             cp_async16(kdst + so, a.kp + off, bytes);
             cp_async16(vdst + so, a.vp + off, bytes);
         }
-        cp_async_commit();
     };
-    if (n_tiles > 0) load_tile(0, 0);
+    // prologue of the ring: tiles that lie wholly inside the committed prefix start before the wait,
+    // the tiles holding this step's new rows (written by the preceding grid) after it
+    int issued = 0;
+    while (issued < STAGES - 1 && issued < n_tiles && k_begin + (issued + 1) * TKEYS <= pos0) {
+        load_tile(issued, issued);
+        cp_async_commit();
+        ++issued;
+    }
+    griddep_wait();
+    griddep_launch_dependents();
+    for (; issued < STAGES - 1; ++issued) {
+        if (issued < n_tiles) load_tile(issued, issued);
+        cp_async_commit();
+    }
 
     // Q rows of this KV head's group, scaled, as (hi, lo) bf16 in swizzled shared memory
     for (int i = tid; i < GP * (HD / 4); i += THREADS) {
@@ -179,13 +197,10 @@ attn_mma_kernel(const AttnArgs a) {
     const uint32_t qh_base = smem_u32(Qh), ql_base = smem_u32(Ql);
 
     for (int tile = 0; tile < n_tiles; ++tile) {
-        const int stage = tile & 1;
-        if (tile + 1 < n_tiles) {
-            load_tile(tile + 1, stage ^ 1);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
+        const int stage = tile % STAGES;
+        if (tile + STAGES - 1 < n_tiles) load_tile(tile + STAGES - 1, (tile + STAGES - 1) % STAGES);
+        cp_async_commit();
+        cp_async_wait<STAGES - 1>();             // tile `tile` has landed
         __syncthreads();
         if (warp < n_slabs) {
             const int k0 = k_begin + tile * TKEYS;
@@ -300,26 +315,44 @@ attn_mma_kernel(const AttnArgs a) {
     if (!s_last) return;
     __threadfence();
 
-    // merge the splits of this (sequence, KV head) in index order
+    // merge the splits of this (sequence, KV head) in index order; the Q area of shared memory is free now
+    float* s_w = reinterpret_cast<float*>(sm);                 // [splits][GP]: row maximum, then the split's weight
+    float* s_l = s_w + a.splits * GP;                          // [splits][GP]: row sum
     const size_t slot0 = ((size_t)b * a.n_kv + kh) * a.splits;
+    for (int i = tid; i < a.splits * G; i += THREADS) {
+        const int sidx = i / G, rho = i % G;
+        const float2 ml = __ldcg(&a.ml_part[(slot0 + sidx) * GP + rho]);
+        s_w[sidx * GP + rho] = ml.x;
+        s_l[sidx * GP + rho] = ml.y;
+    }
+    __syncthreads();
+    for (int rho = tid; rho < G; rho += THREADS) {
+        float mstar = -INFINITY;
+        for (int sidx = 0; sidx < a.splits; ++sidx) mstar = fmaxf(mstar, s_w[sidx * GP + rho]);
+        float den = 0.f;
+        for (int sidx = 0; sidx < a.splits; ++sidx) {
+            const float mv = s_w[sidx * GP + rho];
+            const float w = mv == -INFINITY ? 0.f : exp2f(mv - mstar);
+            den += w * s_l[sidx * GP + rho];
+            s_l[sidx * GP + rho] = w;
+        }
+        const float inv = den > 0.f ? 1.0f / den : 0.f;
+        for (int sidx = 0; sidx < a.splits; ++sidx) s_w[sidx * GP + rho] = s_l[sidx * GP + rho] * inv;
+    }
+    __syncthreads();
     for (int i = tid; i < G * (HD / 4); i += THREADS) {
         const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
         const int hl = rho / R, rr = rho % R;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rr < rows) {
-            float mstar = -INFINITY;
-            for (int s = 0; s < a.splits; ++s) mstar = fmaxf(mstar, __ldcg(&a.ml_part[(slot0 + s) * GP + rho]).x);
-            float den = 0.f;
-            for (int s = 0; s < a.splits; ++s) {
-                const float2 ml = __ldcg(&a.ml_part[(slot0 + s) * GP + rho]);
-                if (ml.x == -INFINITY) continue;
-                const float w = exp2f(ml.x - mstar);
-                den += w * ml.y;
-                const float4 ov = __ldcg(reinterpret_cast<const float4*>(a.o_part + ((slot0 + s) * GP + rho) * HD + d4));
-                acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+#pragma unroll 4
+            for (int sidx = 0; sidx < a.splits; ++sidx) {
+                const float w = s_w[sidx * GP + rho];
+                if (w != 0.f) {                                // a split without visible keys wrote no O
+                    const float4 ov = __ldcg(reinterpret_cast<const float4*>(a.o_part + ((slot0 + sidx) * GP + rho) * HD + d4));
+                    acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+                }
             }
-            const float inv = 1.0f / den;
-            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
         }
         const int m = b * R + rr;
         const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
@@ -335,7 +368,7 @@ attn_mma_kernel(const AttnArgs a) {
 template <int HD, int NW>
 tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
     constexpr int GP = NW * 16;
-    const size_t smem = (size_t)2 * GP * HD * 2 + (size_t)4 * TKEYS * HD * 2;
+    const size_t smem = (size_t)2 * GP * HD * 2 + (size_t)2 * Ring<HD>::STAGES * TKEYS * HD * 2;
     static bool done[64] = {false};
     int dev = 0;
     TASC_CUDA_TRY(cudaGetDevice(&dev));
@@ -373,7 +406,7 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, float* scratch, unsigned int* counters,
                                  int B, int R, int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream) {
     const int G = (n_q / n_kv) * R;
-    if (G > 128 || (hd != 32 && hd != 64 && hd != 128)) return TASC_EINVAL;
+    if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 16) return TASC_EINVAL;
     const int GP = attention_mma_row_pad(G);
     AttnArgs a;
     a.q = qbuf; a.kp = k_pages; a.vp = v_pages; a.block_table = block_table;

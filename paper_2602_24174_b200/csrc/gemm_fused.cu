@@ -11,9 +11,10 @@
 //
 // Split-K.  The narrow matrices of small models give few 128-row tiles, so a cluster of S CTAs shares
 // one output tile and splits the k-range.  Each CTA copies its accumulator to its own shared memory;
-// after a cluster barrier CTA r sums, in fixed rank order, the S copies of its 1/S share of the token
-// columns (ld.shared::cluster) and runs the epilogue for them.  No partial sum reaches global memory,
-// no atomics, and the result does not depend on timing.
+// after a cluster barrier CTA r reads, for its 1/S share of the token columns, the S copies
+// (ld.shared::cluster, all issued before the first is used), adds them in rank order and runs the
+// epilogue for those columns.  No partial sum reaches global memory, there are no atomics, and the
+// result does not depend on timing.
 //
 // RMSNorm without a row-wide pass.  The producer of a normalised input writes x * gain (as hi/lo)
 // and, per 128-feature tile, the row's partial sum of squares; the consumer GEMM multiplies its
@@ -42,6 +43,14 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int THREADS = 192;
 constexpr int LM_SMEM = 4 * 256 * 8;
 constexpr int MAX_DYN_SMEM = 226 * 1024;      // 227 KB per CTA minus the kernel's static shared memory
+
+#ifdef TASC_TIMELINE
+// Development aid, compiled only with -DTASC_TIMELINE: cycle stamps of the phases of every CTA.
+__device__ long long g_timeline[4096][16];
+#define TL(slot) do { if (cta_lin < 4096) g_timeline[cta_lin][slot] = clock64() - tl0; } while (0)
+#else
+#define TL(slot) do { } while (0)
+#endif
 
 __device__ __forceinline__ float4 shfl_xor4(float4 v, int d) {
     float4 r;
@@ -82,6 +91,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int BN = a.BN, stages = a.stages, TB = a.TB;
     const uint32_t b_stage_bytes = (uint32_t)BN * BK * 2;
     const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+    float* xch = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes);          // [TB][128] this CTA's partial tile
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.data_bytes);
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8u * stages;
@@ -89,7 +99,6 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * stages + 1);
     float* s_inv = reinterpret_cast<float*>(bars + 2 * stages + 2);                       // [128]
     unsigned long long* s_arg = reinterpret_cast<unsigned long long*>(s_inv + 128);       // [4][256], LM head only
-    float* red = reinterpret_cast<float*>(smem);                                          // [TB][128], reuses the ring
 
     const int S = (int)cluster_nctarank();
     const int rank = (int)cluster_ctarank();
@@ -100,27 +109,55 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int f0 = out_tile * (EPI == EPI_SWIGLU ? 64 : BM);   // first output feature of the tile
     const int m0 = m_tile * BN;                                // first row of the tile in the activation buffer
     const int t0 = m_tile * TB;                                // first token of the tile
+    int valid = a.M - t0;                                      // token columns in use
+    valid = valid > TB ? TB : valid;
+    const int per = (valid + S - 1) / S;                       // token columns reduced and finished by each CTA of the cluster
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef TASC_TIMELINE
+    const long long tl0 = clock64();
+    const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+#endif
     uint32_t ncols = 32;
     while ((int)ncols < BN) ncols <<= 1;
     __shared__ int s_fail;              // a bounded wait ran out somewhere in this CTA
     auto fail = [&]() { set_status(a.status, TASC_ETIMEOUT); s_fail = 1; };
 
-    if (threadIdx.x == 0) {
-        s_fail = 0;
-        for (int s = 0; s < stages; ++s) {
-            mbar_init(bar_full + 8u * s, 1);
-            mbar_init(bar_empty + 8u * s, 1);
+    const uint64_t pol_w = policy_evict_first();   // weights are read once per step
+    const uint64_t pol_x = policy_evict_last();    // token rows are re-read by every CTA
+    auto load_w = [&](int i, uint32_t dstA, uint32_t bar) {
+        const int kc = (kb_begin + i) * BK;
+        if (EPI == EPI_SWIGLU) {                   // 64 gate rows, then the 64 matching up rows
+            tma_load_2d_hint(dstA, &tmW, kc, f0, bar, pol_w);
+            tma_load_2d_hint(dstA + A_STAGE_BYTES / 2, &tmW, kc, a.N + f0, bar, pol_w);
+        } else {
+            tma_load_2d_hint(dstA, &tmW, kc, f0, bar, pol_w);
         }
-        mbar_init(bar_acc, 1);
-        fence_barrier_init();
-    }
-    if (warp == 4 && lane == 0) {
-        tma_prefetch_desc(&tmW);
-        tma_prefetch_desc(&tmX);
-    }
-    if (warp == 5) {
+    };
+    const int pre = n_kb < stages ? n_kb : stages;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            s_fail = 0;
+            for (int s = 0; s < stages; ++s) {
+                mbar_init(bar_full + 8u * s, 1);
+                mbar_init(bar_empty + 8u * s, 1);
+            }
+            mbar_init(bar_acc, 1);
+            fence_barrier_init();
+            tma_prefetch_desc(&tmW);
+            tma_prefetch_desc(&tmX);
+            // The weights of the first stages depend on no earlier kernel: their loads start before the
+            // rest of the CTA is set up and before the preceding grid has finished.
+            for (int i = 0; i < pre; ++i) {
+                const uint32_t dstA = smem_u32(smem + (size_t)i * stage_bytes);
+                mbar_expect_tx_only(bar_full + 8u * i, A_STAGE_BYTES);
+                load_w(i, dstA, bar_full + 8u * i);
+            }
+            TL(1);
+        }
+        __syncwarp();
+    } else if (warp == 5) {
         tmem_alloc(smem_u32(tmem_slot), ncols);
         tmem_relinquish();
     }
@@ -128,29 +165,13 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) TL(0);
 
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            const uint64_t pol_w = policy_evict_first();   // weights are read once per step
-            const uint64_t pol_x = policy_evict_last();    // token rows are re-read by every CTA
-            auto load_w = [&](int i, uint32_t dstA, uint32_t bar) {
-                const int kc = (kb_begin + i) * BK;
-                if (EPI == EPI_SWIGLU) {                   // 64 gate rows, then the 64 matching up rows
-                    tma_load_2d_hint(dstA, &tmW, kc, f0, bar, pol_w);
-                    tma_load_2d_hint(dstA + A_STAGE_BYTES / 2, &tmW, kc, a.N + f0, bar, pol_w);
-                } else {
-                    tma_load_2d_hint(dstA, &tmW, kc, f0, bar, pol_w);
-                }
-            };
-            // weights of the first stages do not depend on the preceding grid: start them now
-            const int pre = n_kb < stages ? n_kb : stages;
-            for (int i = 0; i < pre; ++i) {
-                const uint32_t dstA = smem_u32(smem + (size_t)i * stage_bytes);
-                mbar_expect_tx_only(bar_full + 8u * i, A_STAGE_BYTES);
-                load_w(i, dstA, bar_full + 8u * i);
-            }
             griddep_wait();
+            TL(2);
             for (int i = 0; i < pre; ++i) {
                 const uint32_t dstB = smem_u32(smem + (size_t)i * stage_bytes) + A_STAGE_BYTES;
                 mbar_expect_tx(bar_full + 8u * i, b_stage_bytes);
@@ -166,6 +187,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 tma_load_2d_hint(dstA + A_STAGE_BYTES, &tmX, (kb_begin + i) * BK, m0, bar_full + 8u * s, pol_x);
             }
             griddep_launch_dependents();
+            TL(3);
         }
         __syncwarp();
     } else if (warp == 5) {
@@ -177,6 +199,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 const int s = i % stages;
                 const uint32_t round = (uint32_t)(i / stages);
                 if (!mbar_wait(bar_full + 8u * s, round & 1u)) { fail(); ok = false; break; }
+                if (i == 0) TL(4);
                 tc_fence_after();
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                 const uint32_t sb = sa + A_STAGE_BYTES;
@@ -189,6 +212,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 umma_commit(bar_empty + 8u * s);
             }
             if (ok) umma_commit(bar_acc);
+            TL(5);
         }
         __syncwarp();
     } else {
@@ -205,45 +229,56 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
         bool have = n_kb > 0;
         if (have && !mbar_wait(bar_acc, 0)) { fail(); have = false; }
+        if (threadIdx.x == 0) TL(6);
         tc_fence_after();
         asm volatile("bar.sync 1, 128;" ::: "memory");          // s_inv visible to the four epilogue warps
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-        for (int c = 0; c < TB / 16; ++c) {
-            uint32_t r[16];
+        const int fl = warp * 32 + lane;                        // this thread's feature (TMEM lane) within the tile
+        for (int c = 0; c < TB; c += 32) {
+            const bool wide = c + 32 <= TB;                     // TB is a multiple of 16
+            uint32_t r[32];
             if (have) {
-                tmem_ld16(lane_base + (uint32_t)(c * 16), r);
-                if (a.pair) {
-                    uint32_t r2[16];
-                    tmem_ld16(lane_base + (uint32_t)(TB + c * 16), r2);
+                if (wide) {
+                    uint32_t r2[32];
+                    tmem_ld32(lane_base + (uint32_t)c, r);
+                    tmem_ld32(lane_base + (uint32_t)(TB + c), r2);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
                 } else {
+                    uint32_t q[16], q2[16];
+                    tmem_ld16(lane_base + (uint32_t)c, q);
+                    tmem_ld16(lane_base + (uint32_t)(TB + c), q2);
                     tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(q[j]) + __uint_as_float(q2[j]));
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) r[j] = 0u;
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
             }
             if (EPI == EPI_LM) {
-                const int f = f0 + warp * 32 + lane;
+                const int f = f0 + fl;
                 const bool f_ok = f < a.N;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int n = c * 16 + j;
-                    const float v = __uint_as_float(r[j]);
-                    const uint32_t key = f_ok ? float_key(v) : 0u;
-                    const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
-                    if (lane == 0) {
-                        const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
-                        s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
+                for (int j = 0; j < 32; ++j) {
+                    if (j < 16 || wide) {
+                        const int n = c + j;
+                        const float v = __uint_as_float(r[j]);
+                        const uint32_t key = f_ok ? float_key(v) : 0u;
+                        const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
+                        const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
+                        if (lane == 0) {
+                            const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
+                            s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
+                        }
+                        if (a.logits && f_ok && t0 + n < a.M) a.logits[(size_t)(t0 + n) * a.N + f] = v * s_inv[n];
                     }
-                    if (a.logits && f_ok && t0 + n < a.M) a.logits[(size_t)(t0 + n) * a.N + f] = v * s_inv[n];
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) red[(c * 16 + j) * BM + warp * 32 + lane] = __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j)
+                    if (j < 16 || wide) xch[(c + j) * BM + fl] = __uint_as_float(r[j]);
             }
         }
         if (EPI == EPI_LM) {
@@ -259,25 +294,32 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             }
         }
     }
+    if (threadIdx.x == 0) TL(7);
     tc_fence_before();
+    // every CTA's partial tile is in its shared memory (release / acquire at cluster scope)
     cluster_arrive();
     cluster_wait();
+    if (threadIdx.x == 0) TL(8);
 
     if (warp < 4 && EPI != EPI_LM) {
-        // ------------------------------------------------------------ epilogue, part 2: this CTA's share of the token columns
-        int valid = a.M - t0;
-        valid = valid > TB ? TB : valid;
-        const int per = (valid + S - 1) / S;
-        const int c0 = rank * per;
-        const int c1 = c0 + per < valid ? c0 + per : valid;
-        const uint32_t red_addr = smem_u32(red);
-        for (int t = c0 + warp; t < c1; t += 4) {
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            const uint32_t off = red_addr + (uint32_t)((t * BM + 4 * lane) * 4);
-            for (int s = 0; s < S; ++s) {
-                const float4 p = ld_cluster_f4(cluster_map(off, (uint32_t)s));
-                acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
-            }
+        // ------------------------------------------------------------ epilogue, part 2: sum the S partial copies of this CTA's columns, finish them
+        int count = valid - rank * per;
+        count = count < 0 ? 0 : (count > per ? per : count);
+        const uint32_t xch_addr = smem_u32(xch) + (uint32_t)(lane * 16);
+        uint32_t peer[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) peer[s] = cluster_map(xch_addr, (uint32_t)(s < S ? s : 0));
+        for (int tl = warp; tl < count; tl += 4) {
+            const int t = rank * per + tl;
+            // all S remote reads are issued before the first is used; they are added in rank order
+            float4 part[8];
+#pragma unroll
+            for (int s = 0; s < 8; ++s)
+                if (s < S) part[s] = ld_cluster_f4(peer[s] + (uint32_t)t * (BM * 4));
+            float4 acc = part[0];
+#pragma unroll
+            for (int s = 1; s < 8; ++s)
+                if (s < S) { acc.x += part[s].x; acc.y += part[s].y; acc.z += part[s].z; acc.w += part[s].w; }
             const int m = t0 + t;
             if (EPI == EPI_PLAIN) {
                 const float sc = a.ssq_in ? s_inv[t] : 1.0f;
@@ -358,7 +400,8 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             }
         }
     }
-    // peers may still be reading this CTA's shared memory
+    if (threadIdx.x == 0) TL(9);
+    // peers may still be reading this CTA's staging buffer
     cluster_arrive();
     cluster_wait();
     if (s_fail && warp == 4 && lane == 0) {
@@ -373,6 +416,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         tc_fence_after();
         tmem_dealloc(tmem_base, ncols);
     }
+    if (threadIdx.x == 0) TL(10);
 }
 
 template <int EPI>
@@ -433,12 +477,13 @@ FusedPlan plan_fused(int M, int N, int K, int epi) {
     while (ncols < p.BN) ncols <<= 1;
     // Up to 128 accumulator columns: about 100 KB so that two CTAs (or this grid and the next one's
     // prologue) share an SM; wider tiles take one CTA per SM and a deeper ring.
-    const int budget = ncols <= 128 ? 96 * 1024 : 192 * 1024;
+    const int xch_bytes = p.TB * BM * 4;                        // the CTA's partial tile for the split-K exchange, not aliased with the ring
+    const int budget = (ncols <= 128 ? 100 * 1024 : 216 * 1024) - xch_bytes;
     int st = budget / stage_bytes;
     st = std::max(2, std::min(st, 8));
     st = std::min(st, std::max(2, kb_per));
     p.stages = st;
-    p.data_bytes = std::max(st * stage_bytes, p.TB * BM * 4);
+    p.data_bytes = st * stage_bytes + xch_bytes;
     int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4 + (epi == EPI_LM ? LM_SMEM : 0);
     // TMEM columns held by co-resident CTAs must never exceed 512, or CTAs of different clusters can
     // block each other's allocation while waiting at a cluster barrier: shared memory limits residency.
@@ -460,5 +505,11 @@ tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap
         default: return TASC_EINVAL;
     }
 }
+
+#ifdef TASC_TIMELINE
+extern "C" int tasc_debug_timeline(long long* out, int n_ctas) {
+    return (int)cudaMemcpyFromSymbol(out, g_timeline, (size_t)n_ctas * 16 * sizeof(long long));
+}
+#endif
 
 }  // namespace tasc
