@@ -85,12 +85,13 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     w.o = L.take<uint8_t>(base, act_rows * m->q_dim * esz);
     w.act = L.take<uint8_t>(base, act_rows * d.d_ff * esz);
     const size_t n_max = std::max<size_t>({(size_t)m->qkv_rows, (size_t)2 * d.d_ff, (size_t)d.d_model});
-    w.partial_bytes = std::max(MIN_PARTIAL_BYTES, M * n_max * sizeof(float));
+    // split-K partial sums in global memory are used by the float32 model only
+    w.partial_bytes = d.dtype == TASC_F32 ? std::max(MIN_PARTIAL_BYTES, M * n_max * sizeof(float)) : ALIGN;
     w.partials = L.take<float>(base, w.partial_bytes / sizeof(float));
     const int splits_max = attention_splits(B, d.n_kv_heads, 1 << 30);
     const size_t att_bytes = d.dtype == TASC_F32
         ? attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max)
-        : attention_mma_scratch_bytes(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * TASC_MAX_ROWS, splits_max);
+        : attention_mma_scratch_bytes(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * TASC_MAX_ROWS, 16);
     w.att_scratch = L.take<float>(base, att_bytes / sizeof(float));
     w.ssq_slots = (d.d_model + 127) / 128;
     w.ssq = L.take<float>(base, M * w.ssq_slots);
@@ -201,7 +202,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
-    const int att_splits = attention_splits(B, d.n_kv_heads, max_ctx);
+    const int att_splits = attention_mma_splits(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * R, max_ctx);
     const int TB = gemm_token_tile(M, true);
     const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
     CUtensorMap tm_h, tm_o, tm_act;

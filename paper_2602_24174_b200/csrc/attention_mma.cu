@@ -13,7 +13,7 @@
 // probabilities P are float32 values carried as hi + lo bf16 pairs, two MMAs each, so the only rounding
 // in the attention is the KV cache's own.  Softmax statistics and O are float32.
 //
-// Merge: each CTA writes its unnormalised O and (max, sum) to scratch and takes a ticket; the CTA
+// Merge (only when the key range is split): each CTA writes its unnormalised O and (max, sum) to scratch and takes a ticket; the CTA
 // that draws the last ticket of a (sequence, KV head) merges the splits in index order and writes the
 // result as (hi, lo) bf16 rows in the layout the O-projection GEMM loads.  Which CTA merges depends on
 // timing, what it computes does not.
@@ -100,6 +100,9 @@ attn_mma_kernel(const AttnArgs a) {
 
     const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef TASC_TIMELINE
+    struct LogAtExit { unsigned long long t0, ta, tb; __device__ ~LogAtExit() { if (threadIdx.x == 0) ctalog_put(t0, ta, tb, 10); } } log_at_exit{global_ns(), 0, 0};
+#endif
     const int g = a.n_q / a.n_kv, R = a.R;
     const int G = g * R;
     const int qd = a.n_q * HD;
@@ -131,6 +134,13 @@ attn_mma_kernel(const AttnArgs a) {
     const int k_end = min(total, k_begin + chunk);
     const int n_tiles = k_begin < k_end ? (k_end - k_begin + TKEYS - 1) / TKEYS : 0;
     const int n_slabs = (G + 15) / 16;
+    // With few query rows the spare warps take every other key tile: warp group `grp` (n_slabs warps,
+    // one 16-row slab each) handles tiles grp, grp + ng, ...; the groups' results are merged in shared memory.
+    const int ng = (STAGES >= 4 && NW / n_slabs >= 2) ? 2 : 1;
+    const int slab = warp % n_slabs, grp = warp / n_slabs;
+    const bool computes = grp < ng;
+    const int n_super = (n_tiles + ng - 1) / ng;                 // iterations of ng tiles
+    const int super_stages = STAGES / ng;
 
     auto load_tile = [&](int tile, int stage) {
         const int k0 = k_begin + tile * TKEYS;
@@ -154,20 +164,24 @@ attn_mma_kernel(const AttnArgs a) {
             cp_async16(vdst + so, a.vp + off, bytes);
         }
     };
+    auto load_super = [&](int sup) {                             // the ng tiles of iteration `sup`, one commit group
+        for (int j = 0; j < ng; ++j)
+            if (sup * ng + j < n_tiles) load_tile(sup * ng + j, (sup % super_stages) * ng + j);
+        cp_async_commit();
+    };
     // prologue of the ring: tiles that lie wholly inside the committed prefix start before the wait,
     // the tiles holding this step's new rows (written by the preceding grid) after it
     int issued = 0;
-    while (issued < STAGES - 1 && issued < n_tiles && k_begin + (issued + 1) * TKEYS <= pos0) {
-        load_tile(issued, issued);
-        cp_async_commit();
+    while (issued < super_stages - 1 && issued < n_super && k_begin + (issued + 1) * ng * TKEYS <= pos0) {
+        load_super(issued);
         ++issued;
     }
     griddep_wait();
+#ifdef TASC_TIMELINE
+    log_at_exit.ta = global_ns();
+#endif
     griddep_launch_dependents();
-    for (; issued < STAGES - 1; ++issued) {
-        if (issued < n_tiles) load_tile(issued, issued);
-        cp_async_commit();
-    }
+    for (; issued < super_stages - 1; ++issued) load_super(issued);   // commits an empty group past the end
 
     // Q rows of this KV head's group, scaled, as (hi, lo) bf16 in swizzled shared memory
     for (int i = tid; i < GP * (HD / 4); i += THREADS) {
@@ -187,7 +201,7 @@ attn_mma_kernel(const AttnArgs a) {
     }
 
     // per-thread rows of the slab: r0 = lane / 4 and r0 + 8
-    const int rho0 = warp * 16 + (lane >> 2), rho1 = rho0 + 8;
+    const int rho0 = slab * 16 + (lane >> 2), rho1 = rho0 + 8;
     const int lim0 = (rho0 < G && rho0 % R < rows) ? min(pos0 + rho0 % R, k_end - 1) : -1;   // last visible key
     const int lim1 = (rho1 < G && rho1 % R < rows) ? min(pos0 + rho1 % R, k_end - 1) : -1;
     float o[HD / 8][4];
@@ -196,13 +210,14 @@ attn_mma_kernel(const AttnArgs a) {
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
     const uint32_t qh_base = smem_u32(Qh), ql_base = smem_u32(Ql);
 
-    for (int tile = 0; tile < n_tiles; ++tile) {
-        const int stage = tile % STAGES;
-        if (tile + STAGES - 1 < n_tiles) load_tile(tile + STAGES - 1, (tile + STAGES - 1) % STAGES);
-        cp_async_commit();
-        cp_async_wait<STAGES - 1>();             // tile `tile` has landed
+    for (int sup = 0; sup < n_super; ++sup) {
+        if (sup + super_stages - 1 < n_super) load_super(sup + super_stages - 1);
+        else cp_async_commit();
+        if (ng == 1) cp_async_wait<STAGES - 1>(); else cp_async_wait<STAGES / 2 - 1>();   // iteration `sup` has landed
         __syncthreads();
-        if (warp < n_slabs) {
+        const int tile = sup * ng + grp;
+        if (computes && tile < n_tiles) {
+            const int stage = (sup % super_stages) * ng + grp;
             const int k0 = k_begin + tile * TKEYS;
             const uint32_t kbase = smem_u32(Kt + stage * TILE_BYTES), vbase = smem_u32(Vt + stage * TILE_BYTES);
             float s[8][4];
@@ -212,7 +227,7 @@ attn_mma_kernel(const AttnArgs a) {
 #pragma unroll
             for (int ks = 0; ks < HD / 16; ++ks) {
                 uint32_t qh[4], ql[4];
-                const uint32_t qo = swz<HD>(warp * 16 + (mi & 1) * 8 + li, ks * 2 + (mi >> 1));
+                const uint32_t qo = swz<HD>(slab * 16 + (mi & 1) * 8 + li, ks * 2 + (mi >> 1));
                 ldsm_x4(qh_base + qo, qh);
                 ldsm_x4(ql_base + qo, ql);
 #pragma unroll
@@ -282,14 +297,68 @@ attn_mma_kernel(const AttnArgs a) {
         }
         __syncthreads();
     }
-
-    // this split's partial result
-    const size_t slot = ((size_t)b * a.n_kv + kh) * a.splits + sp;
-    if (warp < n_slabs) {
+#ifdef TASC_TIMELINE
+    log_at_exit.tb = global_ns();
+#endif
+    if (computes) {
         l_run[0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[0], 1);
         l_run[0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[0], 2);
         l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], 1);
         l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], 2);
+    }
+    if (ng == 2) {
+        // second warp group -> shared memory (the K/V ring is idle) -> first group folds it into its own state
+        float* xg = reinterpret_cast<float*>(Kt) + (size_t)(slab * 32 + lane) * (HD / 2 + 4);
+        if (computes && grp == 1) {
+#pragma unroll
+            for (int i = 0; i < HD / 8; ++i) { xg[4 * i] = o[i][0]; xg[4 * i + 1] = o[i][1]; xg[4 * i + 2] = o[i][2]; xg[4 * i + 3] = o[i][3]; }
+            xg[HD / 2] = m_run[0]; xg[HD / 2 + 1] = m_run[1]; xg[HD / 2 + 2] = l_run[0]; xg[HD / 2 + 3] = l_run[1];
+        }
+        __syncthreads();
+        if (grp == 0) {
+            const float om0 = xg[HD / 2], om1 = xg[HD / 2 + 1], ol0 = xg[HD / 2 + 2], ol1 = xg[HD / 2 + 3];
+            const float mn0 = fmaxf(m_run[0], om0), mn1 = fmaxf(m_run[1], om1);
+            const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+            const float sa0 = exp2f(m_run[0] - mu0), sb0 = exp2f(om0 - mu0), sa1 = exp2f(m_run[1] - mu1), sb1 = exp2f(om1 - mu1);
+#pragma unroll
+            for (int i = 0; i < HD / 8; ++i) {
+                o[i][0] = o[i][0] * sa0 + xg[4 * i] * sb0;     o[i][1] = o[i][1] * sa0 + xg[4 * i + 1] * sb0;
+                o[i][2] = o[i][2] * sa1 + xg[4 * i + 2] * sb1; o[i][3] = o[i][3] * sa1 + xg[4 * i + 3] * sb1;
+            }
+            l_run[0] = l_run[0] * sa0 + ol0 * sb0; l_run[1] = l_run[1] * sa1 + ol1 * sb1;
+            m_run[0] = mn0; m_run[1] = mn1;
+        }
+    }
+    const bool writer = computes && grp == 0;                  // holds the CTA's result for its slab
+
+    if (a.splits == 1) {
+        // the whole key range was here: normalise and write the rows straight to the O-projection's input
+        if (writer) {
+            const float inv0 = l_run[0] > 0.f ? 1.0f / l_run[0] : 0.f, inv1 = l_run[1] > 0.f ? 1.0f / l_run[1] : 0.f;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int rho = half ? rho1 : rho0;
+                if (rho >= G) continue;
+                const int hl = rho / R, rr = rho % R;
+                const float inv = (rr < rows) ? (half ? inv1 : inv0) : 0.f;
+                const int m = b * R + rr;
+                const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
+                const size_t col = (size_t)(kh * g + hl) * HD + 2 * (lane & 3);
+#pragma unroll
+                for (int nt = 0; nt < HD / 8; ++nt) {
+                    uint32_t h, l;
+                    pack_hilo(o[nt][2 * half] * inv, o[nt][2 * half + 1] * inv, h, l);
+                    *reinterpret_cast<uint32_t*>(a.out + row * qd + col + nt * 8) = h;
+                    *reinterpret_cast<uint32_t*>(a.out + (row + a.TB) * qd + col + nt * 8) = l;
+                }
+            }
+        }
+        return;
+    }
+
+    // this split's partial result
+    const size_t slot = ((size_t)b * a.n_kv + kh) * a.splits + sp;
+    if (writer) {
         if (n_tiles > 0) {
             float* op0 = a.o_part + (slot * GP + rho0) * HD + 2 * (lane & 3);
             float* op1 = a.o_part + (slot * GP + rho1) * HD + 2 * (lane & 3);
@@ -395,6 +464,25 @@ tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
 }  // namespace
 
 int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
+
+// Key-range splits per (sequence, KV head), from a small cost model in microseconds: a CTA needs about
+// 1.5 us to start plus one tile time per iteration (its warp groups take `ng` tiles per iteration), all CTAs
+// run in waves of about two per SM, and splitting adds the scratch round trip and the merge (about 3.5 us).
+int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx) {
+    const int n_tiles = (max_ctx + TKEYS - 1) / TKEYS;
+    const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;
+    const int ng = (hd < 128 && nw / n_slabs >= 2) ? 2 : 1;
+    const float t_tile = hd >= 128 ? 0.9f : (hd >= 64 ? 0.45f : 0.3f);
+    int best = 1;
+    float best_cost = 1e30f;
+    for (int s = 1; s <= 16 && s <= n_tiles; ++s) {
+        const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
+        const int waves = (B * n_kv * s + 295) / 296;
+        const float cost = waves * (1.5f + iters * t_tile) + (s > 1 ? 3.5f : 0.f);
+        if (cost < best_cost - 1e-6f) { best_cost = cost; best = s; }
+    }
+    return best;
+}
 
 size_t attention_mma_scratch_bytes(int B, int n_kv, int hd, int G, int n_splits) {
     const size_t slots = (size_t)B * n_kv * n_splits * attention_mma_row_pad(G);

@@ -31,6 +31,8 @@
 #include "kernels.h"
 
 #include <algorithm>
+#include <map>
+#include <mutex>
 
 namespace tasc {
 
@@ -92,6 +94,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const uint32_t b_stage_bytes = (uint32_t)BN * BK * 2;
     const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
     float* xch = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes);          // [TB][128] this CTA's partial tile
+    float* fin = reinterpret_cast<float*>(smem);                                          // [per][128] reduced columns (the ring is idle by then)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.data_bytes);
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8u * stages;
@@ -116,6 +119,8 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #ifdef TASC_TIMELINE
     const long long tl0 = clock64();
+    const unsigned long long g_t0 = global_ns();
+    __shared__ unsigned long long g_ta, g_tb;
     const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
 #endif
     uint32_t ncols = 32;
@@ -218,6 +223,9 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     } else {
         // ------------------------------------------------------------ epilogue, part 1: accumulator -> shared memory
         griddep_wait();
+#ifdef TASC_TIMELINE
+        if (threadIdx.x == 0) g_ta = global_ns();
+#endif
         if (EPI == EPI_QKV || EPI == EPI_SWIGLU || EPI == EPI_LM || (EPI == EPI_PLAIN && a.ssq_in)) {
             for (int t = threadIdx.x; t < TB; t += 128) {
                 const int m = t0 + t;
@@ -230,6 +238,9 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         bool have = n_kb > 0;
         if (have && !mbar_wait(bar_acc, 0)) { fail(); have = false; }
         if (threadIdx.x == 0) TL(6);
+#ifdef TASC_TIMELINE
+        if (threadIdx.x == 0) g_tb = global_ns();
+#endif
         tc_fence_after();
         asm volatile("bar.sync 1, 128;" ::: "memory");          // s_inv visible to the four epilogue warps
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
@@ -305,21 +316,34 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // ------------------------------------------------------------ epilogue, part 2: sum the S partial copies of this CTA's columns, finish them
         int count = valid - rank * per;
         count = count < 0 ? 0 : (count > per ? per : count);
-        const uint32_t xch_addr = smem_u32(xch) + (uint32_t)(lane * 16);
-        uint32_t peer[8];
+        if (S > 1) {
+            // pull: all S remote reads of a column are issued before the first is used, then added in rank order
+            const uint32_t xch_addr = smem_u32(xch) + (uint32_t)(lane * 16);
+            uint32_t peer[8];
 #pragma unroll
-        for (int s = 0; s < 8; ++s) peer[s] = cluster_map(xch_addr, (uint32_t)(s < S ? s : 0));
+            for (int s = 0; s < 8; ++s) peer[s] = cluster_map(xch_addr, (uint32_t)(s < S ? s : 0));
+            for (int tl = warp; tl < count; tl += 4) {
+                const uint32_t toff = (uint32_t)(rank * per + tl) * (BM * 4);
+                float4 part[8];
+#pragma unroll
+                for (int s = 0; s < 8; ++s)
+                    if (s < S) part[s] = ld_cluster_f4(peer[s] + toff);
+                float4 acc = part[0];
+#pragma unroll
+                for (int s = 1; s < 8; ++s)
+                    if (s < S) { acc.x += part[s].x; acc.y += part[s].y; acc.z += part[s].z; acc.w += part[s].w; }
+                *reinterpret_cast<float4*>(fin + (size_t)tl * BM + 4 * lane) = acc;     // read back by the same lane below
+            }
+        }
+    }
+    // this CTA has finished reading its peers' shared memory; they may leave while it runs the epilogue
+    cluster_arrive();
+    if (warp < 4 && EPI != EPI_LM) {
+        int count = valid - rank * per;
+        count = count < 0 ? 0 : (count > per ? per : count);
         for (int tl = warp; tl < count; tl += 4) {
             const int t = rank * per + tl;
-            // all S remote reads are issued before the first is used; they are added in rank order
-            float4 part[8];
-#pragma unroll
-            for (int s = 0; s < 8; ++s)
-                if (s < S) part[s] = ld_cluster_f4(peer[s] + (uint32_t)t * (BM * 4));
-            float4 acc = part[0];
-#pragma unroll
-            for (int s = 1; s < 8; ++s)
-                if (s < S) { acc.x += part[s].x; acc.y += part[s].y; acc.z += part[s].z; acc.w += part[s].w; }
+            const float4 acc = *reinterpret_cast<const float4*>((S > 1 ? fin + (size_t)tl * BM : xch + (size_t)t * BM) + 4 * lane);
             const int m = t0 + t;
             if (EPI == EPI_PLAIN) {
                 const float sc = a.ssq_in ? s_inv[t] : 1.0f;
@@ -331,14 +355,14 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 }
             } else if (EPI == EPI_QKV) {
                 const float sc = s_inv[t];
-                acc.x *= sc; acc.y *= sc; acc.z *= sc; acc.w *= sc;
+                const float4 sacc = make_float4(acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc);
                 const int hd = a.hd, half = hd >> 1;
-                const float4 partner = shfl_xor4(acc, half >> 2);
+                const float4 partner = shfl_xor4(sacc, half >> 2);
                 const int f = f0 + 4 * lane;
                 const int qd = a.n_q * hd, kvd = a.n_kv * hd;
                 int pos = a.row_pos[m];
                 if (pos >= a.max_positions) { set_status(a.status, TASC_EINVAL); pos = -1; }
-                float v[4] = {acc.x, acc.y, acc.z, acc.w};
+                float v[4] = {sacc.x, sacc.y, sacc.z, sacc.w};
                 if (f < qd + kvd && pos >= 0) {
                     const int i = f % hd;
                     const float4* cs = reinterpret_cast<const float4*>(a.rope + (size_t)pos * half + (i % half));
@@ -401,8 +425,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
     }
     if (threadIdx.x == 0) TL(9);
-    // peers may still be reading this CTA's staging buffer
-    cluster_arrive();
+    // peers may still be reading this CTA's partial tile
     cluster_wait();
     if (s_fail && warp == 4 && lane == 0) {
         // after a timeout: give this CTA's own tile loads that may still be in flight a bounded time to land
@@ -417,11 +440,13 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         tmem_dealloc(tmem_base, ncols);
     }
     if (threadIdx.x == 0) TL(10);
+#ifdef TASC_TIMELINE
+    if (threadIdx.x == 0) ctalog_put(g_t0, g_ta, g_tb, EPI);
+#endif
 }
 
 template <int EPI>
-tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const FusedArgs& a, const FusedPlan& p, int kind,
-                       cudaStream_t stream) {
+tasc_status prepare_epi() {
     static bool attr_done[64] = {false};
     int dev = 0;
     TASC_CUDA_TRY(cudaGetDevice(&dev));
@@ -430,6 +455,56 @@ tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const Fus
         TASC_CUDA_TRY(cudaFuncSetAttribute(gemm_fused_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM));
         attr_done[dev] = true;
     }
+    return TASC_OK;
+}
+
+// Clusters of S CTAs with `smem` bytes each that the device can hold at once (0 if the query fails).
+template <int EPI>
+int max_active_clusters(int S, int smem) {
+    if (prepare_epi<EPI>() != TASC_OK) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)S, 1, 1);
+    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)S;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_fused_kernel<EPI>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return n;
+}
+
+int max_active_clusters_any(int epi, int S, int smem) {
+    static std::mutex mu;
+    static std::map<long long, int> cache;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    const long long key = (((long long)dev * 8 + epi) * 32 + S) * (1ll << 20) + smem;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    int n = 0;
+    switch (epi) {
+        case EPI_PLAIN:  n = max_active_clusters<EPI_PLAIN>(S, smem); break;
+        case EPI_QKV:    n = max_active_clusters<EPI_QKV>(S, smem); break;
+        case EPI_RESID:  n = max_active_clusters<EPI_RESID>(S, smem); break;
+        case EPI_SWIGLU: n = max_active_clusters<EPI_SWIGLU>(S, smem); break;
+        case EPI_LM:     n = max_active_clusters<EPI_LM>(S, smem); break;
+        default: break;
+    }
+    cache[key] = n;
+    return n;
+}
+
+template <int EPI>
+tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const FusedArgs& a, const FusedPlan& p, int kind,
+                       cudaStream_t stream) {
+    tasc_status pst = prepare_epi<EPI>();
+    if (pst != TASC_OK) return pst;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.S, (unsigned)p.out_tiles, (unsigned)p.m_tiles);
     cfg.blockDim = dim3(THREADS, 1, 1);
@@ -470,25 +545,32 @@ FusedPlan plan_fused(int M, int N, int K, int epi) {
         S = std::min(S, 8);
         S = std::min(S, p.num_kb);
     }
-    p.S = S;
-    const int kb_per = (p.num_kb + S - 1) / S;
     const int stage_bytes = A_STAGE_BYTES + p.BN * BK * 2;
     int ncols = 32;
     while (ncols < p.BN) ncols <<= 1;
-    // Up to 128 accumulator columns: about 100 KB so that two CTAs (or this grid and the next one's
-    // prologue) share an SM; wider tiles take one CTA per SM and a deeper ring.
     const int xch_bytes = p.TB * BM * 4;                        // the CTA's partial tile for the split-K exchange, not aliased with the ring
-    const int budget = (ncols <= 128 ? 100 * 1024 : 216 * 1024) - xch_bytes;
-    int st = budget / stage_bytes;
-    st = std::max(2, std::min(st, 8));
-    st = std::min(st, std::max(2, kb_per));
-    p.stages = st;
-    p.data_bytes = st * stage_bytes + xch_bytes;
-    int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4 + (epi == EPI_LM ? LM_SMEM : 0);
-    // TMEM columns held by co-resident CTAs must never exceed 512, or CTAs of different clusters can
-    // block each other's allocation while waiting at a cluster barrier: shared memory limits residency.
-    smem = std::max(smem, ncols * 454 + 1);
-    p.smem_bytes = std::min(smem, MAX_DYN_SMEM);
+    for (;; --S) {
+        p.S = S;
+        const int kb_per = (p.num_kb + S - 1) / S;
+        // Up to 128 accumulator columns: about 100 KB so that two CTAs (or this grid and the next one's
+        // prologue) share an SM; wider tiles take one CTA per SM and a deeper ring.
+        const int budget = (ncols <= 128 ? 100 * 1024 : 216 * 1024) - xch_bytes;
+        int st = budget / stage_bytes;
+        st = std::max(2, std::min(st, 8));
+        st = std::min(st, std::max(2, kb_per));
+        p.stages = st;
+        p.data_bytes = st * stage_bytes + xch_bytes;
+        int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4 + (epi == EPI_LM ? LM_SMEM : 0);
+        // TMEM columns held by co-resident CTAs must never exceed 512, or CTAs of different clusters can
+        // block each other's allocation while waiting at a cluster barrier: shared memory limits residency.
+        smem = std::max(smem, ncols * 454 + 1);
+        p.smem_bytes = std::min(smem, MAX_DYN_SMEM);
+        if (S == 1) break;
+        // All clusters of the grid should be resident at once: a second, nearly empty wave doubles the
+        // kernel's time.  (Clusters occupy whole groups of SMs inside a GPC, so fewer fit than SMs / S.)
+        const int fit = max_active_clusters_any(epi, S, p.smem_bytes);
+        if (fit <= 0 || tiles <= fit) break;
+    }
     return p;
 }
 
@@ -507,6 +589,17 @@ tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap
 }
 
 #ifdef TASC_TIMELINE
+__device__ CtaRec g_ctalog[1 << 18];
+__device__ unsigned int g_ctalog_n;
+extern "C" int tasc_debug_ctalog(void* out, int max_recs, int reset) {
+    unsigned int n = 0;
+    if (cudaMemcpyFromSymbol(&n, g_ctalog_n, sizeof(n)) != cudaSuccess) return -1;
+    if (n > (1u << 18)) n = 1u << 18;
+    if ((int)n > max_recs) n = (unsigned int)max_recs;
+    if (n && cudaMemcpyFromSymbol(out, g_ctalog, (size_t)n * sizeof(CtaRec)) != cudaSuccess) return -1;
+    if (reset) { const unsigned int z = 0; cudaMemcpyToSymbol(g_ctalog_n, &z, sizeof(z)); }
+    return (int)n;
+}
 extern "C" int tasc_debug_timeline(long long* out, int n_ctas) {
     return (int)cudaMemcpyFromSymbol(out, g_timeline, (size_t)n_ctas * 16 * sizeof(long long));
 }

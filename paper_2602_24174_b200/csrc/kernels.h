@@ -163,5 +163,6 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, float* scratch, unsigned int* counters,
                                  int B, int R, int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream);
 size_t attention_mma_scratch_bytes(int B, int n_kv, int hd, int G, int n_splits);
+int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx);     // 1..16
 
 }  // namespace tasc
