@@ -4,7 +4,7 @@
 // The kernel is bound by streaming K and V from HBM once; the tensor cores only have to keep up with
 // that stream, which a float32 SIMT formulation cannot do beyond a few sequences.  A CTA owns one
 // (sequence, KV head, key range): the key range of a sequence is split over several CTAs because the
-// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a 3-4 stage cp.async pipeline
+// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a 4-8 stage cp.async pipeline
 // (16-byte vectors, every page of a KV head is one contiguous run) into XOR-swizzled shared memory;
 // warp w computes the 16-row slab w of S = Q K^T and O += P V with mma.sync m16n8k16 (ldmatrix
 // fragments, V through ldmatrix.trans) and keeps an online softmax per row in registers.
@@ -61,7 +61,7 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -80,8 +80,9 @@ __device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32
     lo = (uint32_t)__bfloat16_as_ushort(lx) | ((uint32_t)__bfloat16_as_ushort(ly) << 16);
 }
 
-// ring depth of the K/V tile pipeline: enough bytes in flight per CTA to cover the memory latency
-template <int HD> struct Ring { static constexpr int STAGES = HD >= 128 ? 3 : 4; };
+// Ring depth of the K/V tile pipeline.  A CTA streams its key range alone, so the bytes it keeps in flight
+// (ring depth x 8-32 KB per tile) over the memory latency are its bandwidth: 100-190 KB of tiles per CTA.
+template <int HD, int NW> struct Ring { static constexpr int STAGES = HD >= 128 ? (NW > 4 ? 4 : 5) : 8; };
 
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32)
@@ -90,18 +91,20 @@ attn_mma_kernel(const AttnArgs a) {
     constexpr int CH = HD / 8;                   // 16-byte chunks per row
     constexpr int THREADS = NW * 32;
     constexpr int TILE_BYTES = TKEYS * HD * 2;
-    constexpr int STAGES = Ring<HD>::STAGES;
+    constexpr int STAGES = Ring<HD, NW>::STAGES;
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t* Qh = sm;
     uint8_t* Ql = Qh + GP * HD * 2;
     uint8_t* Kt = Ql + GP * HD * 2;              // [STAGES][TKEYS][HD]
     uint8_t* Vt = Kt + STAGES * TILE_BYTES;      // [STAGES][TKEYS][HD]
     __shared__ int s_last;
+    constexpr int MAX_STAGED_PAGES = 1024;
+    __shared__ int s_pages[MAX_STAGED_PAGES];
 
     const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef TASC_TIMELINE
-    struct LogAtExit { unsigned long long t0, ta, tb; __device__ ~LogAtExit() { if (threadIdx.x == 0) ctalog_put(t0, ta, tb, 10); } } log_at_exit{global_ns(), 0, 0};
+    struct LogAtExit { unsigned long long t0, ta, tb, tc, td, te, tf; __device__ ~LogAtExit() { if (threadIdx.x == 0) ctalog_put(t0, ta, tb, 10, tc, td, te, tf); } } log_at_exit{global_ns(), 0, 0, 0, 0, 0, 0};
 #endif
     const int g = a.n_q / a.n_kv, R = a.R;
     const int G = g * R;
@@ -142,26 +145,45 @@ attn_mma_kernel(const AttnArgs a) {
     const int n_super = (n_tiles + ng - 1) / ng;                 // iterations of ng tiles
     const int super_stages = STAGES / ng;
 
+    // Page ids of this CTA's key range, staged once: the tile loads then need no dependent global read.
+    const int pg_lo = k_begin / a.page_size;
+    const int n_pg = n_tiles > 0 ? (k_end - 1) / a.page_size - pg_lo + 1 : 0;
+    const bool pages_staged = n_pg <= MAX_STAGED_PAGES;
+    if (pages_staged) {
+        for (int i = tid; i < n_pg; i += THREADS) {
+            const int pslot = pg_lo + i;
+            int page = -1;
+            if (pslot < a.max_pages) page = a.block_table[(size_t)b * a.max_pages + pslot];
+            s_pages[i] = (page >= 0 && page < a.n_pages) ? page : -1;      // ids outside the pool read as zeros, never as memory
+        }
+        __syncthreads();
+    }
+    // One row of the tile per TPR threads: a page lookup, then the thread's share of the row's 16-byte chunks.
+    constexpr int TPR = THREADS / TKEYS, CPT = CH / TPR;
     auto load_tile = [&](int tile, int stage) {
-        const int k0 = k_begin + tile * TKEYS;
+        const int row = tid / TPR, c0 = (tid % TPR) * CPT;
+        const int key = k_begin + tile * TKEYS + row;
         const uint32_t kdst = smem_u32(Kt + stage * TILE_BYTES), vdst = smem_u32(Vt + stage * TILE_BYTES);
-        for (int i = tid; i < TKEYS * CH; i += THREADS) {
-            const int row = i / CH, c = i % CH;
-            const int key = k0 + row;
-            size_t off = 0;
-            int bytes = 0;
-            if (key < k_end) {
-                const int pslot = key / a.page_size;
-                int page = -1;
-                if (pslot < a.max_pages) page = a.block_table[(size_t)b * a.max_pages + pslot];
-                if (page >= 0 && page < a.n_pages) {       // ids outside the pool read as zeros, never as memory
-                    off = (((size_t)page * a.n_kv + kh) * a.page_size + key % a.page_size) * HD + c * 8;
-                    bytes = 16;
-                }
+        size_t off = 0;
+        int bytes = 0;
+        if (key < k_end) {
+            const int pslot = key / a.page_size;
+            int page = -1;
+            if (pages_staged) page = s_pages[pslot - pg_lo];
+            else if (pslot < a.max_pages) {
+                page = a.block_table[(size_t)b * a.max_pages + pslot];
+                if (page >= a.n_pages) page = -1;
             }
-            const uint32_t so = swz<HD>(row, c);
-            cp_async16(kdst + so, a.kp + off, bytes);
-            cp_async16(vdst + so, a.vp + off, bytes);
+            if (page >= 0) {
+                off = (((size_t)page * a.n_kv + kh) * a.page_size + key % a.page_size) * HD;
+                bytes = 16;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+            const uint32_t so = swz<HD>(row, c0 + j);
+            cp_async16(kdst + so, a.kp + off + (c0 + j) * 8, bytes);
+            cp_async16(vdst + so, a.vp + off + (c0 + j) * 8, bytes);
         }
     };
     auto load_super = [&](int sup) {                             // the ng tiles of iteration `sup`, one commit group
@@ -183,15 +205,24 @@ attn_mma_kernel(const AttnArgs a) {
     griddep_launch_dependents();
     for (; issued < super_stages - 1; ++issued) load_super(issued);   // commits an empty group past the end
 
-    // Q rows of this KV head's group, scaled, as (hi, lo) bf16 in swizzled shared memory
-    for (int i = tid; i < GP * (HD / 4); i += THREADS) {
+    // Q rows of this KV head's group, scaled, as (hi, lo) bf16 in swizzled shared memory.  All global reads
+    // are issued before the first conversion so that their latencies overlap.
+    constexpr int NQ = GP * (HD / 4) / THREADS;
+    float4 qv[NQ];
+#pragma unroll
+    for (int j = 0; j < NQ; ++j) {
+        const int i = tid + j * THREADS;
         const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
         const int hl = rho / R, rr = rho % R;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (rho < G && rr < rows) {
-            v = *reinterpret_cast<const float4*>(a.q + (size_t)(b * R + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
-            v.x *= a.scale_log2e; v.y *= a.scale_log2e; v.z *= a.scale_log2e; v.w *= a.scale_log2e;
-        }
+        qv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (rho < G && rr < rows)
+            qv[j] = *reinterpret_cast<const float4*>(a.q + (size_t)(b * R + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
+    }
+#pragma unroll
+    for (int j = 0; j < NQ; ++j) {
+        const int i = tid + j * THREADS;
+        const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
+        const float4 v = make_float4(qv[j].x * a.scale_log2e, qv[j].y * a.scale_log2e, qv[j].z * a.scale_log2e, qv[j].w * a.scale_log2e);
         uint2 h, l;
         pack_hilo(v.x, v.y, h.x, l.x);
         pack_hilo(v.z, v.w, h.y, l.y);
@@ -209,12 +240,20 @@ attn_mma_kernel(const AttnArgs a) {
     for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
     const uint32_t qh_base = smem_u32(Qh), ql_base = smem_u32(Ql);
+#ifdef TASC_TIMELINE
+    log_at_exit.tc = global_ns();
+#endif
 
     for (int sup = 0; sup < n_super; ++sup) {
         if (sup + super_stages - 1 < n_super) load_super(sup + super_stages - 1);
         else cp_async_commit();
         if (ng == 1) cp_async_wait<STAGES - 1>(); else cp_async_wait<STAGES / 2 - 1>();   // iteration `sup` has landed
         __syncthreads();
+#ifdef TASC_TIMELINE
+        if (sup == 0) log_at_exit.td = global_ns();
+        if (sup == 1) log_at_exit.te = global_ns();
+        if (sup == 2) log_at_exit.tf = global_ns();
+#endif
         const int tile = sup * ng + grp;
         if (computes && tile < n_tiles) {
             const int stage = (sup % super_stages) * ng + grp;
@@ -230,14 +269,19 @@ attn_mma_kernel(const AttnArgs a) {
                 const uint32_t qo = swz<HD>(slab * 16 + (mi & 1) * 8 + li, ks * 2 + (mi >> 1));
                 ldsm_x4(qh_base + qo, qh);
                 ldsm_x4(ql_base + qo, ql);
+                // eight independent accumulators between two MMAs on the same one (hi pass, then lo pass)
+                uint32_t kb[4][4];
+#pragma unroll
+                for (int np = 0; np < 4; ++np) ldsm_x4(kbase + swz<HD>(np * 16 + (mi >> 1) * 8 + li, ks * 2 + (mi & 1)), kb[np]);
 #pragma unroll
                 for (int np = 0; np < 4; ++np) {
-                    uint32_t kb[4];
-                    ldsm_x4(kbase + swz<HD>(np * 16 + (mi >> 1) * 8 + li, ks * 2 + (mi & 1)), kb);
-                    mma_bf16(s[2 * np], qh, kb[0], kb[1]);
-                    mma_bf16(s[2 * np], ql, kb[0], kb[1]);
-                    mma_bf16(s[2 * np + 1], qh, kb[2], kb[3]);
-                    mma_bf16(s[2 * np + 1], ql, kb[2], kb[3]);
+                    mma_bf16(s[2 * np], qh, kb[np][0], kb[np][1]);
+                    mma_bf16(s[2 * np + 1], qh, kb[np][2], kb[np][3]);
+                }
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    mma_bf16(s[2 * np], ql, kb[np][0], kb[np][1]);
+                    mma_bf16(s[2 * np + 1], ql, kb[np][2], kb[np][3]);
                 }
             }
             // causal / range mask (only tiles that reach past the committed prefix or the split's end)
@@ -285,13 +329,18 @@ attn_mma_kernel(const AttnArgs a) {
                 pack_hilo(s[2 * kb + 1][0], s[2 * kb + 1][1], ph[2], pl[2]);
                 pack_hilo(s[2 * kb + 1][2], s[2 * kb + 1][3], ph[3], pl[3]);
 #pragma unroll
-                for (int dp = 0; dp < HD / 16; ++dp) {
-                    uint32_t vb[4];
-                    ldsm_x4_trans(vbase + swz<HD>(kb * 16 + (mi & 1) * 8 + li, dp * 2 + (mi >> 1)), vb);
-                    mma_bf16(o[2 * dp], ph, vb[0], vb[1]);
-                    mma_bf16(o[2 * dp], pl, vb[0], vb[1]);
-                    mma_bf16(o[2 * dp + 1], ph, vb[2], vb[3]);
-                    mma_bf16(o[2 * dp + 1], pl, vb[2], vb[3]);
+                for (int dp = 0; dp < HD / 16; dp += 2) {          // four independent accumulators per pass
+                    uint32_t vb0[4], vb1[4];
+                    ldsm_x4_trans(vbase + swz<HD>(kb * 16 + (mi & 1) * 8 + li, dp * 2 + (mi >> 1)), vb0);
+                    ldsm_x4_trans(vbase + swz<HD>(kb * 16 + (mi & 1) * 8 + li, (dp + 1) * 2 + (mi >> 1)), vb1);
+                    mma_bf16(o[2 * dp], ph, vb0[0], vb0[1]);
+                    mma_bf16(o[2 * dp + 1], ph, vb0[2], vb0[3]);
+                    mma_bf16(o[2 * dp + 2], ph, vb1[0], vb1[1]);
+                    mma_bf16(o[2 * dp + 3], ph, vb1[2], vb1[3]);
+                    mma_bf16(o[2 * dp], pl, vb0[0], vb0[1]);
+                    mma_bf16(o[2 * dp + 1], pl, vb0[2], vb0[3]);
+                    mma_bf16(o[2 * dp + 2], pl, vb1[0], vb1[1]);
+                    mma_bf16(o[2 * dp + 3], pl, vb1[2], vb1[3]);
                 }
             }
         }
@@ -437,13 +486,13 @@ attn_mma_kernel(const AttnArgs a) {
 template <int HD, int NW>
 tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
     constexpr int GP = NW * 16;
-    const size_t smem = (size_t)2 * GP * HD * 2 + (size_t)2 * Ring<HD>::STAGES * TKEYS * HD * 2;
+    const size_t smem = (size_t)2 * GP * HD * 2 + (size_t)2 * Ring<HD, NW>::STAGES * TKEYS * HD * 2;
     static bool done[64] = {false};
     int dev = 0;
     TASC_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return TASC_EINVAL;
     if (!done[dev]) {
-        TASC_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<HD, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        TASC_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<HD, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         done[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};

@@ -35,7 +35,7 @@ __device__ __forceinline__ void set_status(int* status, int code) {
 #ifdef TASC_TIMELINE
 // Development aid, compiled only with -DTASC_TIMELINE (and relocatable device code): one record per CTA
 // (start, end, two intermediate stamps on the global nanosecond timer, a tag naming the kernel).
-struct CtaRec { unsigned long long t0, t1, ta, tb; int tag, x, y, z; };
+struct CtaRec { unsigned long long t0, t1, ta, tb, tc, td, te, tf; int tag, x, y, z; };
 extern __device__ CtaRec g_ctalog[1 << 18];
 extern __device__ unsigned int g_ctalog_n;
 __device__ __forceinline__ unsigned long long global_ns() {
@@ -43,9 +43,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ void ctalog_put(unsigned long long t0, unsigned long long ta, unsigned long long tb, int tag) {
+__device__ __forceinline__ void ctalog_put(unsigned long long t0, unsigned long long ta, unsigned long long tb, int tag,
+                                           unsigned long long tc = 0, unsigned long long td = 0, unsigned long long te = 0,
+                                           unsigned long long tf = 0) {
     const unsigned int i = atomicAdd(&g_ctalog_n, 1u);
-    if (i < (1u << 18)) g_ctalog[i] = CtaRec{t0, global_ns(), ta, tb, tag, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z};
+    if (i < (1u << 18)) g_ctalog[i] = CtaRec{t0, global_ns(), ta, tb, tc, td, te, tf, tag, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z};
 }
 #endif
 

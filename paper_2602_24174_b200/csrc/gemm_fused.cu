@@ -120,7 +120,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #ifdef TASC_TIMELINE
     const long long tl0 = clock64();
     const unsigned long long g_t0 = global_ns();
-    __shared__ unsigned long long g_ta, g_tb;
+    __shared__ unsigned long long g_ta, g_tb, g_tc, g_td, g_te, g_tf;
     const int cta_lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
 #endif
     uint32_t ncols = 32;
@@ -140,6 +140,119 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
     };
     const int pre = n_kb < stages ? n_kb : stages;
+
+    // Token columns this CTA reduces and finishes: [rank * per, rank * per + count).
+    int count = valid - rank * per;
+    count = count < 0 ? 0 : (count > per ? per : count);
+    // Global operands of the epilogue of one column (position, rotary factors, KV page, residual row).  The
+    // first NPF columns of every warp are fetched while the MMAs run, so their latency is off the tail.
+    struct Pre { float4 x, cs01, cs23; int pos, page; };
+    constexpr int NPF = 3;
+    constexpr int EW = 6;                       // all six warps reduce and finish columns (column tl belongs to warp tl % 6)
+    auto prefetch = [&](int tl) -> Pre {
+        Pre q;
+        q.x = q.cs01 = q.cs23 = make_float4(0.f, 0.f, 0.f, 0.f);
+        q.pos = -1; q.page = -1;
+        const int m = t0 + rank * per + tl;
+        const int f = f0 + 4 * lane;
+        if (EPI == EPI_QKV) {
+            const int hd = a.hd, half = hd >> 1;
+            const int qd = a.n_q * hd, kvd = a.n_kv * hd;
+            int pos = a.row_pos[m];
+            if (pos >= a.max_positions) { set_status(a.status, TASC_EINVAL); pos = -1; }
+            q.pos = pos;
+            if (pos >= 0 && f < qd + kvd) {
+                const float4* cs = reinterpret_cast<const float4*>(a.rope + (size_t)pos * half + ((f % hd) % half));
+                q.cs01 = cs[0];                                  // (cos, sin) of four consecutive pair indices
+                q.cs23 = cs[1];
+            }
+            if (pos >= 0 && f >= qd && f < qd + 2 * kvd) {
+                const int pslot = pos / a.page_size;
+                if (pslot < a.max_pages) q.page = a.block_table[(size_t)(m / a.R) * a.max_pages + pslot];
+                if (q.page < 0 || q.page >= a.n_pages) { set_status(a.status, TASC_ENOKV); q.page = -1; }
+            }
+        } else if (EPI == EPI_RESID) {
+            if (f < a.N) q.x = *reinterpret_cast<const float4*>(a.x + (size_t)m * a.N + f);
+        }
+        return q;
+    };
+    float4 gain4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto finish = [&](int tl, const Pre& q) {
+        const int t = rank * per + tl;
+        const float4 acc = *reinterpret_cast<const float4*>((S > 1 ? fin + (size_t)tl * BM : xch + (size_t)t * BM) + 4 * lane);
+        const int m = t0 + t;
+        if (EPI == EPI_PLAIN) {
+            const float sc = a.ssq_in ? s_inv[t] : 1.0f;
+            const float v[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int f = f0 + 4 * lane + e;
+                if (f < a.N) a.y[(size_t)m * a.N + f] = v[e];
+            }
+        } else if (EPI == EPI_QKV) {
+            const float sc = s_inv[t];
+            const float4 sacc = make_float4(acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc);
+            const int hd = a.hd, half = hd >> 1;
+            const float4 partner = shfl_xor4(sacc, half >> 2);
+            const int f = f0 + 4 * lane;
+            const int qd = a.n_q * hd, kvd = a.n_kv * hd;
+            const int pos = q.pos;
+            float v[4] = {sacc.x, sacc.y, sacc.z, sacc.w};
+            if (f < qd + kvd && pos >= 0) {
+                const float co[4] = {q.cs01.x, q.cs01.z, q.cs23.x, q.cs23.z};
+                const float si[4] = {q.cs01.y, q.cs01.w, q.cs23.y, q.cs23.w};
+                const float pv[4] = {partner.x, partner.y, partner.z, partner.w};
+                const float sgn = (f % hd) < half ? -1.0f : 1.0f;   // first half: a c - b s; second half: b c + a s
+#pragma unroll
+                for (int e = 0; e < 4; ++e) v[e] = v[e] * co[e] + sgn * pv[e] * si[e];
+            }
+            if (f < qd) {
+                if (pos < 0) { v[0] = v[1] = v[2] = v[3] = 0.f; }
+                *reinterpret_cast<float4*>(a.qbuf + (size_t)m * qd + f) = make_float4(v[0], v[1], v[2], v[3]);
+            } else if (f < qd + 2 * kvd && pos >= 0 && q.page >= 0) {
+                const bool is_k = f < qd + kvd;
+                const int gidx = f - qd - (is_k ? 0 : kvd);
+                const int kh = gidx / hd, i = gidx % hd;
+                __nv_bfloat16* base = is_k ? a.k_pages : a.v_pages;
+                store_bf16x4(base + (((size_t)q.page * a.n_kv + kh) * a.page_size + pos % a.page_size) * hd + i, v);
+            }
+        } else if (EPI == EPI_RESID) {
+            const int f = f0 + 4 * lane;
+            float ss = 0.f;
+            if (f < a.N) {
+                const float4 xv = make_float4(q.x.x + acc.x, q.x.y + acc.y, q.x.z + acc.z, q.x.w + acc.w);
+                *reinterpret_cast<float4*>(a.x + (size_t)m * a.N + f) = xv;
+                ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
+                const float v[4] = {xv.x * gain4.x, xv.y * gain4.y, xv.z * gain4.z, xv.w * gain4.w};
+                const size_t row = (size_t)m_tile * (2 * TB) + t;
+                store_hilo4(a.a_out + row * a.N + f, a.a_out + (row + TB) * a.N + f, v);
+            }
+            ss = warp_sum(ss);
+            if (lane == 0) a.ssq_out[(size_t)m * a.ssq_out_slots + out_tile] = ss;
+        } else if (EPI == EPI_SWIGLU) {
+            const float sc = s_inv[t];
+            const float4 up = shfl_xor4(acc, 16);              // lanes 0-15 hold gate features, 16-31 the up features
+            const int j = f0 + 4 * lane;
+            if (lane < 16 && j < a.N) {
+                const float gv[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
+                const float u[4] = {up.x * sc, up.y * sc, up.z * sc, up.w * sc};
+                float v[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) v[e] = gv[e] / (1.0f + expf(-gv[e])) * u[e];
+                const size_t row = (size_t)m_tile * (2 * TB) + t;
+                store_hilo4(a.a_out + row * a.N + j, a.a_out + (row + TB) * a.N + j, v);
+            }
+        }
+    };
+    Pre pf[NPF];
+    auto late_prefetch = [&]() {                // warps 4 and 5, after their producer / MMA loops
+        if (EPI != EPI_LM) {
+#pragma unroll
+            for (int i = 0; i < NPF; ++i)
+                if (warp + EW * i < count) pf[i] = prefetch(warp + EW * i);
+            if (EPI == EPI_RESID && f0 + 4 * lane < a.N) gain4 = *reinterpret_cast<const float4*>(a.gain + f0 + 4 * lane);
+        }
+    };
 
     if (warp == 4) {
         if (lane == 0) {
@@ -195,6 +308,8 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             TL(3);
         }
         __syncwarp();
+        griddep_wait();                 // every lane reads rows of earlier grids below
+        late_prefetch();
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issue
         if (lane == 0) {
@@ -220,12 +335,20 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             TL(5);
         }
         __syncwarp();
+        griddep_wait();
+        late_prefetch();
     } else {
         // ------------------------------------------------------------ epilogue, part 1: accumulator -> shared memory
         griddep_wait();
 #ifdef TASC_TIMELINE
         if (threadIdx.x == 0) g_ta = global_ns();
 #endif
+        if (EPI != EPI_LM) {
+#pragma unroll
+            for (int i = 0; i < NPF; ++i)
+                if (warp + EW * i < count) pf[i] = prefetch(warp + EW * i);
+            if (EPI == EPI_RESID && f0 + 4 * lane < a.N) gain4 = *reinterpret_cast<const float4*>(a.gain + f0 + 4 * lane);
+        }
         if (EPI == EPI_QKV || EPI == EPI_SWIGLU || EPI == EPI_LM || (EPI == EPI_PLAIN && a.ssq_in)) {
             for (int t = threadIdx.x; t < TB; t += 128) {
                 const int m = t0 + t;
@@ -306,125 +429,63 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
     }
     if (threadIdx.x == 0) TL(7);
+#ifdef TASC_TIMELINE
+    if (threadIdx.x == 0) g_tc = global_ns();
+#endif
     tc_fence_before();
     // every CTA's partial tile is in its shared memory (release / acquire at cluster scope)
     cluster_arrive();
     cluster_wait();
     if (threadIdx.x == 0) TL(8);
+#ifdef TASC_TIMELINE
+    if (threadIdx.x == 0) g_td = global_ns();
+#endif
 
-    if (warp < 4 && EPI != EPI_LM) {
-        // ------------------------------------------------------------ epilogue, part 2: sum the S partial copies of this CTA's columns, finish them
-        int count = valid - rank * per;
-        count = count < 0 ? 0 : (count > per ? per : count);
+    if (EPI != EPI_LM) {
+        // ------------------------------------------------------------ epilogue, part 2: sum the S partial copies of this CTA's columns
         if (S > 1) {
             // pull: all S remote reads of a column are issued before the first is used, then added in rank order
             const uint32_t xch_addr = smem_u32(xch) + (uint32_t)(lane * 16);
             uint32_t peer[8];
 #pragma unroll
             for (int s = 0; s < 8; ++s) peer[s] = cluster_map(xch_addr, (uint32_t)(s < S ? s : 0));
-            for (int tl = warp; tl < count; tl += 4) {
-                const uint32_t toff = (uint32_t)(rank * per + tl) * (BM * 4);
-                float4 part[8];
+            for (int tl = warp; tl < count; tl += 2 * EW) {       // two columns per round: 2 S reads in flight
+                const bool two = tl + EW < count;
+                const uint32_t toff0 = (uint32_t)(rank * per + tl) * (BM * 4), toff1 = toff0 + (uint32_t)EW * (BM * 4);
+                float4 p0[8], p1[8];
 #pragma unroll
                 for (int s = 0; s < 8; ++s)
-                    if (s < S) part[s] = ld_cluster_f4(peer[s] + toff);
-                float4 acc = part[0];
+                    if (s < S) {
+                        p0[s] = ld_cluster_f4(peer[s] + toff0);
+                        if (two) p1[s] = ld_cluster_f4(peer[s] + toff1);
+                    }
+                float4 a0 = p0[0], a1 = p1[0];
 #pragma unroll
                 for (int s = 1; s < 8; ++s)
-                    if (s < S) { acc.x += part[s].x; acc.y += part[s].y; acc.z += part[s].z; acc.w += part[s].w; }
-                *reinterpret_cast<float4*>(fin + (size_t)tl * BM + 4 * lane) = acc;     // read back by the same lane below
+                    if (s < S) {
+                        a0.x += p0[s].x; a0.y += p0[s].y; a0.z += p0[s].z; a0.w += p0[s].w;
+                        a1.x += p1[s].x; a1.y += p1[s].y; a1.z += p1[s].z; a1.w += p1[s].w;
+                    }
+                *reinterpret_cast<float4*>(fin + (size_t)tl * BM + 4 * lane) = a0;      // read back by the same lane below
+                if (two) *reinterpret_cast<float4*>(fin + (size_t)(tl + EW) * BM + 4 * lane) = a1;
             }
         }
     }
+#ifdef TASC_TIMELINE
+    if (threadIdx.x == 0) g_te = global_ns();
+#endif
     // this CTA has finished reading its peers' shared memory; they may leave while it runs the epilogue
     cluster_arrive();
-    if (warp < 4 && EPI != EPI_LM) {
-        int count = valid - rank * per;
-        count = count < 0 ? 0 : (count > per ? per : count);
-        for (int tl = warp; tl < count; tl += 4) {
-            const int t = rank * per + tl;
-            const float4 acc = *reinterpret_cast<const float4*>((S > 1 ? fin + (size_t)tl * BM : xch + (size_t)t * BM) + 4 * lane);
-            const int m = t0 + t;
-            if (EPI == EPI_PLAIN) {
-                const float sc = a.ssq_in ? s_inv[t] : 1.0f;
-                const float v[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
+    if (EPI != EPI_LM) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int f = f0 + 4 * lane + e;
-                    if (f < a.N) a.y[(size_t)m * a.N + f] = v[e];
-                }
-            } else if (EPI == EPI_QKV) {
-                const float sc = s_inv[t];
-                const float4 sacc = make_float4(acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc);
-                const int hd = a.hd, half = hd >> 1;
-                const float4 partner = shfl_xor4(sacc, half >> 2);
-                const int f = f0 + 4 * lane;
-                const int qd = a.n_q * hd, kvd = a.n_kv * hd;
-                int pos = a.row_pos[m];
-                if (pos >= a.max_positions) { set_status(a.status, TASC_EINVAL); pos = -1; }
-                float v[4] = {sacc.x, sacc.y, sacc.z, sacc.w};
-                if (f < qd + kvd && pos >= 0) {
-                    const int i = f % hd;
-                    const float4* cs = reinterpret_cast<const float4*>(a.rope + (size_t)pos * half + (i % half));
-                    const float4 cs01 = cs[0], cs23 = cs[1];        // (cos, sin) of four consecutive pair indices
-                    const float co[4] = {cs01.x, cs01.z, cs23.x, cs23.z};
-                    const float si[4] = {cs01.y, cs01.w, cs23.y, cs23.w};
-                    const float pv[4] = {partner.x, partner.y, partner.z, partner.w};
-                    const float sgn = i < half ? -1.0f : 1.0f;      // first half: a c - b s; second half: b c + a s
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) v[e] = v[e] * co[e] + sgn * pv[e] * si[e];
-                }
-                if (f < qd) {
-                    if (pos < 0) { v[0] = v[1] = v[2] = v[3] = 0.f; }
-                    *reinterpret_cast<float4*>(a.qbuf + (size_t)m * qd + f) = make_float4(v[0], v[1], v[2], v[3]);
-                } else if (f < qd + 2 * kvd && pos >= 0) {
-                    const int b = m / a.R;
-                    const int pslot = pos / a.page_size;
-                    int page = -1;
-                    if (pslot < a.max_pages) page = a.block_table[(size_t)b * a.max_pages + pslot];
-                    if (page < 0 || page >= a.n_pages) {
-                        set_status(a.status, TASC_ENOKV);
-                    } else {
-                        const bool is_k = f < qd + kvd;
-                        const int g = f - qd - (is_k ? 0 : kvd);
-                        const int kh = g / hd, i = g % hd;
-                        __nv_bfloat16* base = is_k ? a.k_pages : a.v_pages;
-                        store_bf16x4(base + (((size_t)page * a.n_kv + kh) * a.page_size + pos % a.page_size) * hd + i, v);
-                    }
-                }
-            } else if (EPI == EPI_RESID) {
-                const int f = f0 + 4 * lane;
-                float ss = 0.f;
-                if (f < a.N) {
-                    float4* xp = reinterpret_cast<float4*>(a.x + (size_t)m * a.N + f);
-                    float4 xv = *xp;
-                    xv.x += acc.x; xv.y += acc.y; xv.z += acc.z; xv.w += acc.w;
-                    *xp = xv;
-                    ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
-                    const float4 g = *reinterpret_cast<const float4*>(a.gain + f);
-                    const float v[4] = {xv.x * g.x, xv.y * g.y, xv.z * g.z, xv.w * g.w};
-                    const size_t row = (size_t)(m / TB) * (2 * TB) + (m % TB);
-                    store_hilo4(a.a_out + row * a.N + f, a.a_out + (row + TB) * a.N + f, v);
-                }
-                ss = warp_sum(ss);
-                if (lane == 0) a.ssq_out[(size_t)m * a.ssq_out_slots + out_tile] = ss;
-            } else if (EPI == EPI_SWIGLU) {
-                const float sc = s_inv[t];
-                const float4 up = shfl_xor4(acc, 16);              // lanes 0-15 hold gate features, 16-31 the up features
-                const int j = f0 + 4 * lane;
-                if (lane < 16 && j < a.N) {
-                    const float g[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
-                    const float u[4] = {up.x * sc, up.y * sc, up.z * sc, up.w * sc};
-                    float v[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) v[e] = g[e] / (1.0f + expf(-g[e])) * u[e];
-                    const size_t row = (size_t)(m / TB) * (2 * TB) + (m % TB);
-                    store_hilo4(a.a_out + row * a.N + j, a.a_out + (row + TB) * a.N + j, v);
-                }
-            }
-        }
+        for (int i = 0; i < NPF; ++i)
+            if (warp + EW * i < count) finish(warp + EW * i, pf[i]);
+        for (int tl = warp + EW * NPF; tl < count; tl += EW) finish(tl, prefetch(tl));
     }
     if (threadIdx.x == 0) TL(9);
+#ifdef TASC_TIMELINE
+    if (threadIdx.x == 0) g_tf = global_ns();
+#endif
     // peers may still be reading this CTA's partial tile
     cluster_wait();
     if (s_fail && warp == 4 && lane == 0) {
@@ -441,7 +502,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     }
     if (threadIdx.x == 0) TL(10);
 #ifdef TASC_TIMELINE
-    if (threadIdx.x == 0) ctalog_put(g_t0, g_ta, g_tb, EPI);
+    if (threadIdx.x == 0) ctalog_put(g_t0, g_ta, g_tb, EPI, g_tc, g_td, g_te, g_tf);
 #endif
 }
 
