@@ -93,14 +93,17 @@ def step_bytes(shape, B, k, ctx_lens):
 
 
 def gemm_bytes_per_step(shape, M):
-    """Algorithmic bytes of all GEMM launches of one step: weights + (hi, lo) activation rows in + float32 rows out."""
+    """Algorithmic bytes of all fused-GEMM launches of one step: every weight matrix once, the (hi, lo) bf16
+    activation rows each launch reads, and what its epilogue writes (q float32 + K/V bf16; residual rows
+    read + written and the next (hi, lo) rows; SiLU*up (hi, lo) rows; nothing for the LM-head argmax)."""
     s = shape
-    mats = [(s.qkv_rows, s.d_model), (s.d_model, s.q_dim), (2 * s.d_ff, s.d_model), (s.d_model, s.d_ff)]
-    total = 0
-    for n, kk in mats:
-        total += s.n_layers * (n * kk * 2 + 2 * M * kk * 2 + M * n * 4)
-    total += s.vocab * s.d_model * 2 + 2 * M * s.d_model * 2          # LM head: argmax epilogue writes no logits
-    return total
+    hilo = lambda cols: 2 * M * cols * 2
+    per_layer = (
+        s.qkv_rows * s.d_model * 2 + hilo(s.d_model) + M * s.q_dim * 4 + M * 2 * s.kv_dim * 2        # QKV + RoPE + KV append
+        + s.d_model * s.q_dim * 2 + hilo(s.q_dim) + 2 * M * s.d_model * 4 + hilo(s.d_model)         # O + residual
+        + 2 * s.d_ff * s.d_model * 2 + hilo(s.d_model) + hilo(s.d_ff)                               # gate/up + SiLU*mul
+        + s.d_model * s.d_ff * 2 + hilo(s.d_ff) + 2 * M * s.d_model * 4 + hilo(s.d_model))          # down + residual
+    return s.n_layers * per_layer + s.vocab * s.d_model * 2 + hilo(s.d_model)
 
 
 # ----------------------------------------------------------------------------------------------- oracle legs
@@ -169,6 +172,8 @@ def main():
     ap.add_argument("--only-timed", action="store_true",
                     help="device-resident timed region only (no per-kernel pass, e2e, generate or CPU legs): the command ncu wraps")
     ap.add_argument("--sweep", action="store_true", help="also report the teacher-forced acceptance sweep (forced a = 0..k)")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step's kernels from the host instead of replaying a CUDA graph")
+    ap.add_argument("--corpus-docs", type=int, default=None, help="build the drafter from the first N corpus documents only")
     args = ap.parse_args()
     cfg = configs.get(args.config)
     B = args.batch
@@ -197,13 +202,13 @@ def main():
     model = b.Model(shape, b.weights_to_device(host_w, shape.dtype, dev), max_positions=cfg.prompt_len + cfg.max_new + 4096,
                     page_size=cfg.page_size)
     del host_w
-    ctoks, coffs = corpus.make_corpus(cfg)
+    ctoks, coffs = corpus.make_corpus(cfg, n_docs=args.corpus_docs)
     drafter = b.tasc_drafter_build(torch.from_numpy(ctoks).to(dev), torch.from_numpy(coffs).to(dev), cfg.n_max, cfg.p_min, shape.vocab)
     prompts_all = corpus.make_prompts(cfg, B * world)
     prompts = prompts_all[rank * B:(rank + 1) * B]
     P = prompts.shape[1]
     total_steps = args.warmup + args.steps
-    stride = P + (total_steps + args.steps + 2) * (k + 1) + k + 2       # timed pass + instrumented pass share one state
+    stride = P + (total_steps + args.steps + 4) * (k + 1) + k + 2       # timed pass + instrumented pass share one state
     if stride > 12288:
         raise SystemExit("too many steps for one token buffer")
     ws = model.new_workspace(B, k, dev)
@@ -242,11 +247,26 @@ def main():
         b.tasc_draft(drafter, tokens, length, k, cfg.lambda_num, cfg.lambda_den, out=drafts)
         return b.tasc_verify_step(model, kvs[2], seqs, drafts, ws)
 
-    # ---- device-resident timing: `value`
+    # ---- device-resident timing: `value`.  One step (draft + verify, ~5 launches per layer) is captured into a
+    # CUDA graph after the warm-up and replayed K times; the state (tokens, lengths, KV) lives on the device,
+    # so the replays decode on exactly as separate launches would.
     tokens, length, kvs, seqs = fresh_state()
     for _ in range(args.warmup):
         one_step(kvs, seqs, tokens, length)
     b.tasc_poll_status(ws)
+    graph, launches_per_step = None, None
+    if not args.no_graph:
+        cap_stream = torch.cuda.Stream(device=dev)
+        cap_stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cap_stream):
+            c0 = sum(b.tasc_launch_counts().values())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=cap_stream):
+                one_step(kvs, seqs, tokens, length)
+            launches_per_step = sum(b.tasc_launch_counts().values()) - c0      # kernels recorded in the graph
+        torch.cuda.current_stream().wait_stream(cap_stream)
+        torch.cuda.synchronize()
+    run_step = (lambda: graph.replay()) if graph is not None else (lambda: one_step(kvs, seqs, tokens, length))
     len0 = length.clone()
     launches0 = sum(b.tasc_launch_counts().values())
     sampler = ClockSampler(local_rank)
@@ -255,11 +275,11 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.steps):
-        one_step(kvs, seqs, tokens, length)
+        run_step()
     ev1.record()
     barrier()
     clocks = sampler.stop()
-    launches = sum(b.tasc_launch_counts().values()) - launches0
+    launches = (launches_per_step * args.steps) if graph is not None else sum(b.tasc_launch_counts().values()) - launches0
     b.tasc_poll_status(ws)
     ms = max_over_ranks(ev0.elapsed_time(ev1))
     committed = float((length - len0).sum().item())
@@ -289,7 +309,7 @@ def main():
     wbytes, kvbytes = step_bytes(shape, B, k, [ctx_mid] * B)
     step_gbs = (wbytes + kvbytes) / (ms / args.steps * 1e-3) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": "gemm_bf16_kernel (tcgen05 + TMA; all projection, MLP and LM-head launches)",
+        "bound": "hbm", "kernel": "gemm_fused_kernel (tcgen05 + TMA, cluster split-K, fused epilogues; 4 launches per layer + LM head)",
         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
         "traffic": None, "peak_source": peaks["source"],
         "bytes_per_launch_avg": gemm_bytes / max(gemm_launches, 1), "us_per_launch_avg": gemm_ms * 1e3 / max(gemm_launches, 1),
@@ -370,6 +390,7 @@ def main():
             "dtype": "bf16" if shape.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": f"config {cfg.index} ({cfg.name}): B={B} per GPU, k={k}, n_max={cfg.n_max}, prompt {P}, "
                                    f"context {int(len0.float().mean().item())}->{int(length.float().mean().item())}, real greedy targets",
+                       "launch": "one CUDA graph replay per step" if graph is not None else "host launches",
                        "l2": "inputs larger than L2: weights %.0f MB are streamed once per step" % (wbytes / 1e6),
                        "parallelism": "replicas only (independent batches per GPU, no collective)" if world > 1 else "single GPU"},
             "mean_committed_per_step": committed_all / (args.steps * B * world),
