@@ -43,7 +43,6 @@ constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int THREADS = 192;
-constexpr int LM_SMEM = 4 * 256 * 8;
 constexpr int MAX_DYN_SMEM = 226 * 1024;      // 227 KB per CTA minus the kernel's static shared memory
 
 #ifdef TASC_TIMELINE
@@ -101,7 +100,6 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const uint32_t bar_acc = bar_full + 16u * stages;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * stages + 1);
     float* s_inv = reinterpret_cast<float*>(bars + 2 * stages + 2);                       // [128]
-    unsigned long long* s_arg = reinterpret_cast<unsigned long long*>(s_inv + 128);       // [4][256], LM head only
 
     const int S = (int)cluster_nctarank();
     const int rank = (int)cluster_ctarank();
@@ -391,41 +389,9 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = 0u;
             }
-            if (EPI == EPI_LM) {
-                const int f = f0 + fl;
-                const bool f_ok = f < a.N;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    if (j < 16 || wide) {
-                        const int n = c + j;
-                        const float v = __uint_as_float(r[j]);
-                        const uint32_t key = f_ok ? float_key(v) : 0u;
-                        const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-                        const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
-                        if (lane == 0) {
-                            const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
-                            s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
-                        }
-                        if (a.logits && f_ok && t0 + n < a.M) a.logits[(size_t)(t0 + n) * a.N + f] = v * s_inv[n];
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (j < 16 || wide) xch[(c + j) * BM + fl] = __uint_as_float(r[j]);
-            }
-        }
-        if (EPI == EPI_LM) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int n = threadIdx.x; n < TB; n += 128) {
-                if (t0 + n < a.M) {
-                    unsigned long long best = s_arg[n];
-                    best = max(best, s_arg[256 + n]);
-                    best = max(best, s_arg[512 + n]);
-                    best = max(best, s_arg[768 + n]);
-                    atomicMax(&a.argmax[t0 + n], best);
-                }
-            }
+            for (int j = 0; j < 32; ++j)
+                if (j < 16 || wide) xch[(c + j) * BM + fl] = __uint_as_float(r[j]);
         }
     }
     if (threadIdx.x == 0) TL(7);
@@ -481,6 +447,27 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         for (int i = 0; i < NPF; ++i)
             if (warp + EW * i < count) finish(warp + EW * i, pf[i]);
         for (int tl = warp + EW * NPF; tl < count; tl += EW) finish(tl, prefetch(tl));
+    } else {
+        // LM head: per token row the largest logit of this 128-feature tile (smallest id on ties), merged
+        // across tiles by an atomic max on the packed (value, id) word; the logits themselves are not stored
+        for (int t = warp; t < valid; t += EW) {
+            const float4 acc = *reinterpret_cast<const float4*>(xch + (size_t)t * BM + 4 * lane);
+            const float v[4] = {acc.x, acc.y, acc.z, acc.w};
+            const int f = f0 + 4 * lane;
+            unsigned long long best = 0ull;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (f + e < a.N) best = max(best, pack_argmax(v[e], (uint32_t)(f + e)));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
+            if (lane == 0) atomicMax(&a.argmax[t0 + t], best);
+            if (a.logits) {
+                const float sc = s_inv[t];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (f + e < a.N) a.logits[(size_t)(t0 + t) * a.N + f + e] = v[e] * sc;
+            }
+        }
     }
     if (threadIdx.x == 0) TL(9);
 #ifdef TASC_TIMELINE
@@ -613,15 +600,17 @@ FusedPlan plan_fused(int M, int N, int K, int epi) {
     for (;; --S) {
         p.S = S;
         const int kb_per = (p.num_kb + S - 1) / S;
-        // Up to 128 accumulator columns: about 100 KB so that two CTAs (or this grid and the next one's
-        // prologue) share an SM; wider tiles take one CTA per SM and a deeper ring.
-        const int budget = (ncols <= 128 ? 100 * 1024 : 216 * 1024) - xch_bytes;
+        // A CTA's streaming rate is its bytes in flight over the memory latency.  A grid of one wave (at most
+        // one CTA per SM anyway) gets a ring of up to 200 KB; a grid of several waves with narrow tiles keeps
+        // about 100 KB per CTA so that two CTAs share an SM and cover each other's start-up and epilogue.
+        const bool one_wave = tiles * S <= 148;
+        const int budget = ((ncols <= 128 && !one_wave) ? 100 * 1024 : 216 * 1024) - xch_bytes;
         int st = budget / stage_bytes;
         st = std::max(2, std::min(st, 8));
         st = std::min(st, std::max(2, kb_per));
         p.stages = st;
         p.data_bytes = st * stage_bytes + xch_bytes;
-        int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4 + (epi == EPI_LM ? LM_SMEM : 0);
+        int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4;
         // TMEM columns held by co-resident CTAs must never exceed 512, or CTAs of different clusters can
         // block each other's allocation while waiting at a cluster barrier: shared memory limits residency.
         smem = std::max(smem, ncols * 454 + 1);
