@@ -89,9 +89,8 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     w.partial_bytes = d.dtype == TASC_F32 ? std::max(MIN_PARTIAL_BYTES, M * n_max * sizeof(float)) : ALIGN;
     w.partials = L.take<float>(base, w.partial_bytes / sizeof(float));
     const int splits_max = attention_splits(B, d.n_kv_heads, 1 << 30);
-    const size_t att_bytes = d.dtype == TASC_F32
-        ? attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max)
-        : attention_mma_scratch_bytes(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * TASC_MAX_ROWS, 16);
+    // split partials in global memory are used by the float32 model only
+    const size_t att_bytes = d.dtype == TASC_F32 ? attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max) : ALIGN;
     w.att_scratch = L.take<float>(base, att_bytes / sizeof(float));
     w.ssq_slots = (d.d_model + 127) / 128;
     w.ssq = L.take<float>(base, M * w.ssq_slots);
@@ -238,8 +237,8 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
         if ((st = launch_gemm_fused(EPI_QKV, &m->tm_qkv[l], &tm_h, a, p_qkv, s)) != TASC_OK) return st;
 
         st = launch_attention_mma(w.q, static_cast<const __nv_bfloat16*>(kvl.k), static_cast<const __nv_bfloat16*>(kvl.v),
-                                  kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, w.att_scratch,
-                                  w.counters, B, R, d.n_q_heads, d.n_kv_heads, d.head_dim, att_splits, s);
+                                  kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, B, R,
+                                  d.n_q_heads, d.n_kv_heads, d.head_dim, att_splits, s);
         if (st != TASC_OK) return st;
 
         a = base;

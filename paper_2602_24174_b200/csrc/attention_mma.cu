@@ -13,10 +13,10 @@
 // probabilities P are float32 values carried as hi + lo bf16 pairs, two MMAs each, so the only rounding
 // in the attention is the KV cache's own.  Softmax statistics and O are float32.
 //
-// Merge (only when the key range is split): each CTA writes its unnormalised O and (max, sum) to scratch and takes a ticket; the CTA
-// that draws the last ticket of a (sequence, KV head) merges the splits in index order and writes the
-// result as (hi, lo) bf16 rows in the layout the O-projection GEMM loads.  Which CTA merges depends on
-// timing, what it computes does not.
+// Merge (only when the key range is split): the splits of one (sequence, KV head) are the CTAs of a
+// thread-block cluster.  Each parks its unnormalised O and (max, sum) in its shared memory; after a cluster
+// barrier CTA r merges every S-th row from the S copies (distributed shared memory reads, rank order) and
+// writes it as (hi, lo) bf16 in the layout the O-projection GEMM loads.  Nothing goes through global memory.
 #include "kernels.h"
 
 namespace tasc {
@@ -36,9 +36,6 @@ struct AttnArgs {
     const int* seq_rows;
     __nv_bfloat16* out;                // (hi, lo) activation buffer, row length n_q * hd
     int TB;
-    float* o_part;                     // [B][n_kv][splits][GP][hd]
-    float2* ml_part;                   // [B][n_kv][splits][GP]
-    unsigned int* counters;            // [B][n_kv], zero between uses
     int R, n_q, n_kv, splits;
     float scale_log2e;
 };
@@ -97,7 +94,6 @@ attn_mma_kernel(const AttnArgs a) {
     uint8_t* Ql = Qh + GP * HD * 2;
     uint8_t* Kt = Ql + GP * HD * 2;              // [STAGES][TKEYS][HD]
     uint8_t* Vt = Kt + STAGES * TILE_BYTES;      // [STAGES][TKEYS][HD]
-    __shared__ int s_last;
     constexpr int MAX_STAGED_PAGES = 1024;
     __shared__ int s_pages[MAX_STAGED_PAGES];
 
@@ -405,72 +401,61 @@ attn_mma_kernel(const AttnArgs a) {
         return;
     }
 
-    // this split's partial result
-    const size_t slot = ((size_t)b * a.n_kv + kh) * a.splits + sp;
+    // The key range was split over the S CTAs of this cluster: every CTA parks its unnormalised rows
+    // (O, running maximum, running sum) in its own shared memory (the K/V ring is idle); after a cluster
+    // barrier CTA r merges the rows rho = r, r + S, ... from all S copies, in rank order, and writes them.
+    constexpr int XS = HD + 4;                                 // floats per parked row: O[HD], max, sum, pad
+    float* xo = reinterpret_cast<float*>(Kt);
+    __syncthreads();                                           // the warp groups' exchange area is inside the ring too
     if (writer) {
-        if (n_tiles > 0) {
-            float* op0 = a.o_part + (slot * GP + rho0) * HD + 2 * (lane & 3);
-            float* op1 = a.o_part + (slot * GP + rho1) * HD + 2 * (lane & 3);
+        float* r0p = xo + (size_t)rho0 * XS + 2 * (lane & 3);
+        float* r1p = xo + (size_t)rho1 * XS + 2 * (lane & 3);
 #pragma unroll
-            for (int nt = 0; nt < HD / 8; ++nt) {
-                *reinterpret_cast<float2*>(op0 + nt * 8) = make_float2(o[nt][0], o[nt][1]);
-                *reinterpret_cast<float2*>(op1 + nt * 8) = make_float2(o[nt][2], o[nt][3]);
-            }
+        for (int nt = 0; nt < HD / 8; ++nt) {
+            *reinterpret_cast<float2*>(r0p + nt * 8) = make_float2(o[nt][0], o[nt][1]);
+            *reinterpret_cast<float2*>(r1p + nt * 8) = make_float2(o[nt][2], o[nt][3]);
         }
         if ((lane & 3) == 0) {
-            a.ml_part[slot * GP + rho0] = make_float2(m_run[0], l_run[0]);
-            a.ml_part[slot * GP + rho1] = make_float2(m_run[1], l_run[1]);
+            *reinterpret_cast<float2*>(xo + (size_t)rho0 * XS + HD) = make_float2(m_run[0], l_run[0]);
+            *reinterpret_cast<float2*>(xo + (size_t)rho1 * XS + HD) = make_float2(m_run[1], l_run[1]);
         }
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned int ticket = atomicAdd(&a.counters[b * a.n_kv + kh], 1u);
-        s_last = ticket == (unsigned int)(a.splits - 1);
-        if (s_last) a.counters[b * a.n_kv + kh] = 0u;        // ready for the next layer
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-
-    // merge the splits of this (sequence, KV head) in index order; the Q area of shared memory is free now
-    float* s_w = reinterpret_cast<float*>(sm);                 // [splits][GP]: row maximum, then the split's weight
-    float* s_l = s_w + a.splits * GP;                          // [splits][GP]: row sum
-    const size_t slot0 = ((size_t)b * a.n_kv + kh) * a.splits;
-    for (int i = tid; i < a.splits * G; i += THREADS) {
-        const int sidx = i / G, rho = i % G;
-        const float2 ml = __ldcg(&a.ml_part[(slot0 + sidx) * GP + rho]);
-        s_w[sidx * GP + rho] = ml.x;
-        s_l[sidx * GP + rho] = ml.y;
-    }
-    __syncthreads();
-    for (int rho = tid; rho < G; rho += THREADS) {
-        float mstar = -INFINITY;
-        for (int sidx = 0; sidx < a.splits; ++sidx) mstar = fmaxf(mstar, s_w[sidx * GP + rho]);
-        float den = 0.f;
-        for (int sidx = 0; sidx < a.splits; ++sidx) {
-            const float mv = s_w[sidx * GP + rho];
-            const float w = mv == -INFINITY ? 0.f : exp2f(mv - mstar);
-            den += w * s_l[sidx * GP + rho];
-            s_l[sidx * GP + rho] = w;
-        }
-        const float inv = den > 0.f ? 1.0f / den : 0.f;
-        for (int sidx = 0; sidx < a.splits; ++sidx) s_w[sidx * GP + rho] = s_l[sidx * GP + rho] * inv;
-    }
-    __syncthreads();
-    for (int i = tid; i < G * (HD / 4); i += THREADS) {
-        const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
+    cluster_arrive();
+    cluster_wait();
+    const int S = a.splits, rank = (int)cluster_ctarank();
+    const uint32_t xo_addr = smem_u32(xo);
+    uint32_t peer[8];
+#pragma unroll
+    for (int sidx = 0; sidx < 8; ++sidx) peer[sidx] = cluster_map(xo_addr, (uint32_t)(sidx < S ? sidx : 0));
+    const int my_rows = rank < G ? (G - rank + S - 1) / S : 0;
+    for (int i = tid; i < my_rows * (HD / 4); i += THREADS) {
+        const int rho = rank + (i / (HD / 4)) * S, d4 = (i % (HD / 4)) * 4;
         const int hl = rho / R, rr = rho % R;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rr < rows) {
-#pragma unroll 4
-            for (int sidx = 0; sidx < a.splits; ++sidx) {
-                const float w = s_w[sidx * GP + rho];
-                if (w != 0.f) {                                // a split without visible keys wrote no O
-                    const float4 ov = __ldcg(reinterpret_cast<const float4*>(a.o_part + ((slot0 + sidx) * GP + rho) * HD + d4));
-                    acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+            float2 ml[8];
+            float4 ov[8];
+#pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx)
+                if (sidx < S) {                                 // all remote reads are issued before the first is used
+                    const uint32_t rowa = peer[sidx] + (uint32_t)(rho * XS) * 4u;
+                    ml[sidx] = ld_cluster_f2(rowa + HD * 4u);
+                    ov[sidx] = ld_cluster_f4(rowa + (uint32_t)d4 * 4u);
                 }
-            }
+            float mstar = -INFINITY;
+#pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx)
+                if (sidx < S) mstar = fmaxf(mstar, ml[sidx].x);
+            float den = 0.f;
+#pragma unroll
+            for (int sidx = 0; sidx < 8; ++sidx)
+                if (sidx < S && ml[sidx].x != -INFINITY) {      // a split without visible keys holds zeros
+                    const float w = exp2f(ml[sidx].x - mstar);
+                    den += w * ml[sidx].y;
+                    acc.x += w * ov[sidx].x; acc.y += w * ov[sidx].y; acc.z += w * ov[sidx].z; acc.w += w * ov[sidx].w;
+                }
+            const float inv = den > 0.f ? 1.0f / den : 0.f;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
         }
         const int m = b * R + rr;
         const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
@@ -481,6 +466,9 @@ attn_mma_kernel(const AttnArgs a) {
         *reinterpret_cast<uint2*>(a.out + row * qd + col) = h;
         *reinterpret_cast<uint2*>(a.out + (row + a.TB) * qd + col) = l;
     }
+    // peers may still be reading this CTA's parked rows
+    cluster_arrive();
+    cluster_wait();
 }
 
 template <int HD, int NW>
@@ -500,11 +488,19 @@ tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
     cfg.blockDim = dim3(NW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
+    int n_at = 1;
+    if (a.splits > 1) {                            // the key-range splits of one (sequence, KV head) form a cluster
+        at[n_at].id = cudaLaunchAttributeClusterDimension;
+        at[n_at].val.clusterDim.x = (unsigned)a.splits;
+        at[n_at].val.clusterDim.y = 1;
+        at[n_at].val.clusterDim.z = 1;
+        ++n_at;
+    }
     cfg.attrs = at;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = n_at;
     ProfScope ps(K_ATT_SPLIT, stream);
     TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_mma_kernel<HD, NW>, a));
     return TASC_OK;
@@ -514,9 +510,9 @@ tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
 
 int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
 
-// Key-range splits per (sequence, KV head), from a small cost model in microseconds: a CTA needs about
-// 1.5 us to start plus one tile time per iteration (its warp groups take `ng` tiles per iteration), all CTAs
-// run in waves of about two per SM, and splitting adds the scratch round trip and the merge (about 3.5 us).
+// Key-range splits per (sequence, KV head), 1..8 (a cluster), from a small cost model in microseconds: a CTA
+// needs about 1.5 us to start plus one tile time per iteration (its warp groups take `ng` tiles per iteration),
+// all CTAs run in waves of about two per SM, and splitting adds the cluster exchange and merge (about 3 us).
 int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx) {
     const int n_tiles = (max_ctx + TKEYS - 1) / TKEYS;
     const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;
@@ -524,36 +520,27 @@ int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx) {
     const float t_tile = hd >= 128 ? 0.9f : (hd >= 64 ? 0.45f : 0.3f);
     int best = 1;
     float best_cost = 1e30f;
-    for (int s = 1; s <= 16 && s <= n_tiles; ++s) {
+    for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
         const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
         const int waves = (B * n_kv * s + 295) / 296;
-        const float cost = waves * (1.5f + iters * t_tile) + (s > 1 ? 3.5f : 0.f);
+        const float cost = waves * (1.5f + iters * t_tile) + (s > 1 ? 3.0f : 0.f);
         if (cost < best_cost - 1e-6f) { best_cost = cost; best = s; }
     }
     return best;
 }
 
-size_t attention_mma_scratch_bytes(int B, int n_kv, int hd, int G, int n_splits) {
-    const size_t slots = (size_t)B * n_kv * n_splits * attention_mma_row_pad(G);
-    return slots * hd * sizeof(float) + slots * sizeof(float2);
-}
-
 tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
                                  const int32_t* block_table, int max_pages, int page_size, long long n_pages,
-                                 const RowPlan& rp, __nv_bfloat16* out, int TB, float* scratch, unsigned int* counters,
-                                 int B, int R, int n_q, int n_kv, int hd, int n_splits, cudaStream_t stream) {
+                                 const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
+                                 int n_splits, cudaStream_t stream) {
     const int G = (n_q / n_kv) * R;
-    if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 16) return TASC_EINVAL;
+    if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 8) return TASC_EINVAL;
     const int GP = attention_mma_row_pad(G);
     AttnArgs a;
     a.q = qbuf; a.kp = k_pages; a.vp = v_pages; a.block_table = block_table;
     a.max_pages = max_pages; a.page_size = page_size; a.n_pages = n_pages;
     a.seq_pos0 = rp.seq_pos0; a.seq_rows = rp.seq_rows;
     a.out = out; a.TB = TB;
-    const size_t slots = (size_t)B * n_kv * n_splits * GP;
-    a.o_part = scratch;
-    a.ml_part = reinterpret_cast<float2*>(scratch + slots * hd);
-    a.counters = counters;
     a.R = R; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits;
     a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
     if (GP == 64) {
