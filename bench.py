@@ -85,6 +85,31 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+# ----------------------------------------------------------------------------------------------- replicas
+# The path does not shard: sequences are independent, so N GPUs run N independent replicas (own prompts,
+# replicated weights and tables) with no data-path collective.  Only the timing is reduced over ranks.
+def shard_prompts(prompts_all, rank: int, per_rank: int):
+    """Rows of the global prompt array that belong to `rank` (per_rank sequences each)."""
+    return prompts_all[rank * per_rank:(rank + 1) * per_rank]
+
+
+def reduce_over_ranks(x: float, op: str, world: int, device) -> float:
+    """max or sum of a scalar over all ranks (identity for one rank)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def whole_job_throughput(units_local: float, ms_local: float, world: int, device) -> tuple:
+    """(units all ranks processed / slowest rank's time, that time in ms)."""
+    ms = reduce_over_ranks(ms_local, "max", world, device)
+    return reduce_over_ranks(units_local, "sum", world, device) / (ms * 1e-3), ms
+
+
 def step_bytes(shape, B, k, ctx_lens):
     """Algorithmic HBM bytes of one verify step: every weight once, every live KV byte once, the new KV rows."""
     wbytes = shape.matmul_params() * 2
@@ -205,7 +230,7 @@ def main():
     ctoks, coffs = corpus.make_corpus(cfg, n_docs=args.corpus_docs)
     drafter = b.tasc_drafter_build(torch.from_numpy(ctoks).to(dev), torch.from_numpy(coffs).to(dev), cfg.n_max, cfg.p_min, shape.vocab)
     prompts_all = corpus.make_prompts(cfg, B * world)
-    prompts = prompts_all[rank * B:(rank + 1) * B]
+    prompts = shard_prompts(prompts_all, rank, B)
     P = prompts.shape[1]
     total_steps = args.warmup + args.steps
     stride = P + (total_steps + args.steps + 4) * (k + 1) + k + 2       # timed pass + instrumented pass share one state
@@ -230,18 +255,10 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_over_ranks(x, "max", world, dev)
 
     def sum_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
+        return reduce_over_ranks(x, "sum", world, dev)
 
     def one_step(kvs, seqs, tokens, length):
         b.tasc_draft(drafter, tokens, length, k, cfg.lambda_num, cfg.lambda_den, out=drafts)

@@ -51,7 +51,6 @@ struct Workspace {
     float* att_scratch;
     float* ssq;                   // [M][ceil(d / 128)] partial sums of squares of the residual rows (bf16 models)
     int ssq_slots;
-    unsigned int* counters;       // [B * n_kv] attention merge tickets
     size_t bytes;
 };
 
@@ -94,7 +93,6 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     w.att_scratch = L.take<float>(base, att_bytes / sizeof(float));
     w.ssq_slots = (d.d_model + 127) / 128;
     w.ssq = L.take<float>(base, M * w.ssq_slots);
-    w.counters = L.take<unsigned int>(base, (size_t)B * d.n_kv_heads);
     w.bytes = L.off;
     return w;
 }
@@ -117,78 +115,41 @@ KvView layer_kv(const tasc_model* m, const tasc_kv* kv, int layer) {
     return KvView{base, base + per};
 }
 
-// One GEMM of the forward: P = X[M][K] * W[N][K]^T as split partials; returns the number of splits.
-template <typename T>
-tasc_status run_gemm(const tasc_model* m, const Workspace& w, const void* X, const CUtensorMap* tmX, const void* W,
-                     const CUtensorMap* tmW, int M, int N, int K, int* splits, unsigned long long* argmax, float* logits,
-                     cudaStream_t s) {
-    if constexpr (sizeof(T) == 4) {
-        (void)m; (void)tmX; (void)tmW;
-        launch_gemm_f32(static_cast<const float*>(X), static_cast<const float*>(W), w.partials, M, N, K, argmax, logits, s);
-        *splits = 1;
-        return TASC_OK;
-    } else {
-        (void)X; (void)W;
-        GemmPlan plan = plan_gemm(M, N, K, w.partial_bytes, true);
-        if (argmax) plan.splits = 1;
-        *splits = plan.splits;
-        return launch_gemm_bf16(tmW, tmX, w.partials, M, N, K, plan, argmax, logits, w.status, s);
-    }
-}
-
-// Forward of M = B * R rows described by w.rp; fills the KV cache; optionally the LM head + argmax.
-template <typename T>
-tasc_status forward(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
-                    cudaStream_t s) {
+// float32 model (the tiny configuration): one launch per stage, float32 SIMT kernels.
+tasc_status forward_f32(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
+                        cudaStream_t s) {
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
     const int att_splits = attention_splits(B, d.n_kv_heads, max_ctx);
-    CUtensorMap tm_h, tm_o, tm_act;
-    int TB = 0;
-    if constexpr (sizeof(T) == 2) {
-        TB = gemm_token_tile(M, true);                      // token tile depends on M only
-        const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
-        tasc_status st;
-        if ((st = encode_tmap_bf16(&tm_h, w.h, rows, d.d_model, 2 * TB)) != TASC_OK) return st;
-        if ((st = encode_tmap_bf16(&tm_o, w.o, rows, m->q_dim, 2 * TB)) != TASC_OK) return st;
-        if ((st = encode_tmap_bf16(&tm_act, w.act, rows, d.d_ff, 2 * TB)) != TASC_OK) return st;
-    }
-    T* h = static_cast<T*>(w.h);
+    float* h = static_cast<float*>(w.h);
     float* q = w.q;
-    T* o = static_cast<T*>(w.o);
-    T* act = static_cast<T*>(w.act);
-    launch_embed_norm<T>(static_cast<const T*>(m->embed), w.rp.row_tok, m->attn_norm[0], d.rms_eps, w.x, h, M, d.d_model, TB, s);
+    float* o = static_cast<float*>(w.o);
+    float* act = static_cast<float*>(w.act);
+    auto gemm = [&](const float* X, const void* W, int N, int K, unsigned long long* argmax, float* lg) {
+        launch_gemm_f32(X, static_cast<const float*>(W), w.partials, M, N, K, argmax, lg, s);
+    };
+    launch_embed_norm<float>(static_cast<const float*>(m->embed), w.rp.row_tok, m->attn_norm[0], d.rms_eps, w.x, h, M, d.d_model, 0, s);
     for (int l = 0; l < d.n_layers; ++l) {
         const KvView kvl = layer_kv(m, kv, l);
-        int sp = 1;
-        tasc_status st;
-        const bool bf = sizeof(T) == 2;
-        st = run_gemm<T>(m, w, h, &tm_h, m->wqkv[l], bf ? &m->tm_qkv[l] : nullptr, M, m->qkv_rows, d.d_model, &sp, nullptr, nullptr, s);
-        if (st != TASC_OK) return st;
-        launch_qkv_rope_append<T>(w.partials, sp, w.rp, m->rope, q, static_cast<T*>(kvl.k), static_cast<T*>(kvl.v),
-                                  kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, M, R, d.n_q_heads,
-                                  d.n_kv_heads, d.head_dim, d.max_positions, w.status, s);
-        launch_attention<T>(q, static_cast<const T*>(kvl.k), static_cast<const T*>(kvl.v), kv->block_table,
-                            kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, w.att_scratch, B, R, d.n_q_heads,
-                            d.n_kv_heads, d.head_dim, att_splits, s);
-        st = run_gemm<T>(m, w, o, &tm_o, m->wo[l], bf ? &m->tm_o[l] : nullptr, M, d.d_model, m->q_dim, &sp, nullptr, nullptr, s);
-        if (st != TASC_OK) return st;
-        launch_residual_norm<T>(w.partials, sp, w.x, m->mlp_norm[l], d.rms_eps, h, M, d.d_model, TB, s);
-        st = run_gemm<T>(m, w, h, &tm_h, m->w_gate_up[l], bf ? &m->tm_gu[l] : nullptr, M, 2 * d.d_ff, d.d_model, &sp, nullptr, nullptr, s);
-        if (st != TASC_OK) return st;
-        launch_silu_mul<T>(w.partials, sp, act, M, d.d_ff, TB, s);
-        st = run_gemm<T>(m, w, act, &tm_act, m->w_down[l], bf ? &m->tm_down[l] : nullptr, M, d.d_model, d.d_ff, &sp, nullptr, nullptr, s);
-        if (st != TASC_OK) return st;
+        gemm(h, m->wqkv[l], m->qkv_rows, d.d_model, nullptr, nullptr);
+        launch_qkv_rope_append<float>(w.partials, 1, w.rp, m->rope, q, static_cast<float*>(kvl.k), static_cast<float*>(kvl.v),
+                                      kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, M, R, d.n_q_heads,
+                                      d.n_kv_heads, d.head_dim, d.max_positions, w.status, s);
+        launch_attention<float>(q, static_cast<const float*>(kvl.k), static_cast<const float*>(kvl.v), kv->block_table,
+                                kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, 0, w.att_scratch, B, R, d.n_q_heads,
+                                d.n_kv_heads, d.head_dim, att_splits, s);
+        gemm(o, m->wo[l], d.d_model, m->q_dim, nullptr, nullptr);
+        launch_residual_norm<float>(w.partials, 1, w.x, m->mlp_norm[l], d.rms_eps, h, M, d.d_model, 0, s);
+        gemm(h, m->w_gate_up[l], 2 * d.d_ff, d.d_model, nullptr, nullptr);
+        launch_silu_mul<float>(w.partials, 1, act, M, d.d_ff, 0, s);
+        gemm(act, m->w_down[l], d.d_model, d.d_ff, nullptr, nullptr);
         const float* next_gain = l + 1 < d.n_layers ? m->attn_norm[l + 1] : m->final_norm;
-        launch_residual_norm<T>(w.partials, sp, w.x, next_gain, d.rms_eps, h, M, d.d_model, TB, s);
+        launch_residual_norm<float>(w.partials, 1, w.x, next_gain, d.rms_eps, h, M, d.d_model, 0, s);
     }
     if (lm_head) {
-        int sp = 1;
         launch_fill_u64(w.argmax, 0ull, M, s);
-        tasc_status st = run_gemm<T>(m, w, h, &tm_h, m->lm_head, sizeof(T) == 2 ? &m->tm_lm : nullptr, M, d.vocab, d.d_model,
-                                     &sp, w.argmax, logits, s);
-        if (st != TASC_OK) return st;
+        gemm(h, m->lm_head, d.vocab, d.d_model, w.argmax, logits);
     }
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;
@@ -266,7 +227,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
 
 tasc_status forward_any(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
                         cudaStream_t s) {
-    return m->desc.dtype == TASC_F32 ? forward<float>(m, kv, w, B, R, lm_head, logits, s)
+    return m->desc.dtype == TASC_F32 ? forward_f32(m, kv, w, B, R, lm_head, logits, s)
                                      : forward_bf16(m, kv, w, B, R, lm_head, logits, s);
 }
 
@@ -282,8 +243,7 @@ tasc_status verify_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_se
                            const int32_t* drafts, int B, int k, const int32_t* forced, int32_t* n_accepted,
                            int32_t* next_token, int32_t* target_tokens, float* logits, cudaStream_t s) {
     const int R = k + 1;
-    launch_rows_verify(w.rp, seqs->tokens, seqs->stride, seqs->len, seqs->stop_len, drafts, B, R, m->desc.vocab, w.status, w.counters,
-                       B * m->desc.n_kv_heads, s);
+    launch_rows_verify(w.rp, seqs->tokens, seqs->stride, seqs->len, seqs->stop_len, drafts, B, R, m->desc.vocab, w.status, s);
     tasc_status st = forward_any(m, kv, w, B, R, true, logits, s);
     if (st != TASC_OK) return st;
     launch_accept(w.argmax, w.rp, drafts, forced, seqs->tokens, seqs->stride, seqs->len, B, R, n_accepted, next_token,
@@ -297,8 +257,7 @@ tasc_status prefill_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_s
     const int R = TASC_MAX_ROWS;
     const int chunks = (std::max(max_len - 1, 0) + R - 1) / R;
     for (int c = 0; c < chunks; ++c) {
-        launch_rows_prefill(w.rp, seqs->tokens, seqs->stride, seqs->len, B, R, c, m->desc.vocab, w.status, w.counters,
-                            B * m->desc.n_kv_heads, s);
+        launch_rows_prefill(w.rp, seqs->tokens, seqs->stride, seqs->len, B, R, c, m->desc.vocab, w.status, s);
         tasc_status st = forward_any(m, kv, w, B, R, false, nullptr, s);
         if (st != TASC_OK) return st;
     }
@@ -518,7 +477,7 @@ extern "C" tasc_status tasc_gemm_bf16(const void* x, const void* wt, float* y, i
     if ((st = encode_tmap_bf16(&tmX, x, M, K, p.BN)) != TASC_OK) return st;
     int* status = static_cast<int*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
-    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, nullptr, nullptr, status, s)) != TASC_OK) return st;
+    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, status, s)) != TASC_OK) return st;
     launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;

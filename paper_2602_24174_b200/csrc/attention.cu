@@ -227,8 +227,5 @@ void launch_attention(const float* qbuf, const T* k_pages, const T* v_pages, con
 
 template void launch_attention<float>(const float*, const float*, const float*, const int32_t*, int, int, long long,
                                       const RowPlan&, float*, int, float*, int, int, int, int, int, int, cudaStream_t);
-template void launch_attention<__nv_bfloat16>(const float*, const __nv_bfloat16*, const __nv_bfloat16*, const int32_t*, int,
-                                              int, long long, const RowPlan&, __nv_bfloat16*, int, float*, int, int, int, int,
-                                              int, int, cudaStream_t);
 
 }  // namespace tasc

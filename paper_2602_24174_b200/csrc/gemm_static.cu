@@ -70,7 +70,7 @@ extern "C" tasc_status tasc_gemm_bf16_static(const void* x, const void* wt, floa
     int* status = device_status ? device_status : reinterpret_cast<int*>(scratch);
     TASC_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));
     float* partials = reinterpret_cast<float*>(scratch + STATUS_BYTES);
-    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, nullptr, nullptr, status, s)) != TASC_OK) return st;
+    if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, status, s)) != TASC_OK) return st;
     launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;

@@ -1,17 +1,12 @@
-// bf16 GEMM for the verify forward on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA.
+// General-purpose bf16 GEMM on the 5th-generation tensor cores (tcgen05 + TMEM), fed by TMA, with split-K
+// partial sums in global memory: the exported building block (tasc_gemm_bf16, tasc_gemm_bf16_static).
+// The verify forward itself runs the fused variant in gemm_fused.cu, which shares this kernel's operand
+// layout and pipeline but reduces split-K inside a cluster and fuses the consumer stage.
 //
-// The verify step multiplies a handful of token rows (M = B * (k+1)) by large weight matrices, so
-// the operands are swapped: the weight tile supplies the 128 rows of the MMA (UMMA M = 128), the
-// token rows are the MMA's N (16..256).  D^T[128 weight rows][BN tokens] accumulates in TMEM in
-// float32.  The kernel is weight-bandwidth bound: each CTA streams a [128 x k-range] slab of W
-// through a multi-stage TMA -> shared-memory ring; split-K spreads a matrix with few row tiles
-// over all SMs.  Partial sums go to global memory and are added in fixed order by the consumer
-// kernels, so results do not depend on scheduling.
-//
-// Paired mode (the forward's activations): a float32 activation v is carried as two bf16 rows,
-// hi = bf16(v) and lo = bf16(v - hi), stored tile by tile as [TB hi rows][TB lo rows] (BN = 2 TB).
-// Both halves go through the same MMA and the epilogue adds accumulator columns j and j + TB, so
-// the product keeps about 16 mantissa bits of the activation at no extra weight traffic.
+// Operands are swapped: the weight tile supplies the 128 rows of the MMA (UMMA M = 128), the token rows
+// are the MMA's N (16..256); D^T[128 weight rows][BN tokens] accumulates in TMEM in float32.  Each CTA
+// streams a [128 x k-range] slab of W through a multi-stage TMA -> shared-memory ring; split-K spreads a
+// matrix with few row tiles over all SMs and the slices are added in fixed order afterwards.
 //
 // Warp roles (192 threads): warps 0-3 epilogue (TMEM lanes 32w..32w+31), warp 4 TMA producer,
 // warp 5 TMEM allocation + MMA issue.  Every wait is bounded; on timeout the CTA records
@@ -30,15 +25,12 @@ constexpr int BK = 64;            // k elements per stage: 64 bf16 = one 128-byt
 constexpr int UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int GEMM_THREADS = 192;
-constexpr int ARGMAX_SMEM = 4 * 256 * 8;
 
 struct GemmArgs {
     float* partials;
     int M, N, K;
     int num_kb, splits, m_tiles, BN, stages;
     int pair;                       // 1: columns j and j + BN/2 of the accumulator belong to the same token
-    unsigned long long* argmax;
-    float* logits;
     int* status;
 };
 
@@ -56,7 +48,6 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     const uint32_t bar_empty = bar_full + 8u * stages;
     const uint32_t bar_acc = bar_full + 16u * stages;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * stages + 1);
-    unsigned long long* s_arg = reinterpret_cast<unsigned long long*>(bars + 2 * stages + 2);   // [4][256]
 
     int bid = blockIdx.x;
     const int m_tile = bid % a.m_tiles; bid /= a.m_tiles;
@@ -161,37 +152,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 16; ++j) r[j] = 0u;
             }
-            if (a.argmax) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int n = c * 16 + j;
-                    const uint32_t key = f_ok ? float_key(__uint_as_float(r[j])) : 0u;
-                    const uint32_t mx = __reduce_max_sync(0xFFFFFFFFu, key);
-                    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == mx);
-                    if (lane == 0) {
-                        const uint32_t id = (uint32_t)(f0 + warp * 32 + (__ffs(who) - 1));
-                        s_arg[warp * 256 + n] = ((unsigned long long)mx << 32) | (unsigned long long)(0xFFFFFFFFu - id);
-                    }
-                    if (a.logits && f_ok && t0 + n < a.M) a.logits[(size_t)(t0 + n) * a.N + f] = __uint_as_float(r[j]);
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int m = t0 + c * 16 + j;
-                    if (f_ok && m < a.M) a.partials[((size_t)split * a.M + m) * a.N + f] = __uint_as_float(r[j]);
-                }
-            }
-        }
-        if (a.argmax) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int n = threadIdx.x; n < TBk; n += 128) {
-                if (t0 + n < a.M) {
-                    unsigned long long best = s_arg[n];
-                    best = max(best, s_arg[256 + n]);
-                    best = max(best, s_arg[512 + n]);
-                    best = max(best, s_arg[768 + n]);
-                    atomicMax(&a.argmax[t0 + n], best);
-                }
+            for (int j = 0; j < 16; ++j) {
+                const int m = t0 + c * 16 + j;
+                if (f_ok && m < a.M) a.partials[((size_t)split * a.M + m) * a.N + f] = __uint_as_float(r[j]);
             }
         }
     }
@@ -220,7 +184,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 int stage_bytes_for(int BN) { return A_STAGE_BYTES + BN * BK * 2; }
-int smem_for(int BN, int stages) { return 1024 + stages * stage_bytes_for(BN) + (2 * stages + 2) * 8 + ARGMAX_SMEM; }
+int smem_for(int BN, int stages) { return 1024 + stages * stage_bytes_for(BN) + (2 * stages + 2) * 8; }
 
 }  // namespace
 
@@ -276,16 +240,14 @@ tasc_status gemm_set_attributes() {
 }
 
 tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, float* partials, int M, int N, int K,
-                             const GemmPlan& plan, unsigned long long* argmax, float* logits, int* status,
-                             cudaStream_t stream) {
+                             const GemmPlan& plan, int* status, cudaStream_t stream) {
     if (M <= 0 || N <= 0 || K <= 0) return TASC_EINVAL;
-    if (argmax && plan.splits != 1) return TASC_EINVAL;
     GemmArgs a;
     a.partials = partials; a.M = M; a.N = N; a.K = K;
     a.num_kb = (K + BK - 1) / BK; a.splits = plan.splits; a.m_tiles = plan.m_tiles; a.BN = plan.BN; a.stages = plan.stages; a.pair = plan.pair;
-    a.argmax = argmax; a.logits = logits; a.status = status;
+    a.status = status;
     const int grid = plan.out_tiles * plan.splits * plan.m_tiles;
-    ProfScope ps(argmax ? K_GEMM_LM : K_GEMM, stream);
+    ProfScope ps(K_GEMM, stream);
     gemm_bf16_kernel<<<grid, GEMM_THREADS, plan.smem_bytes, stream>>>(*tmW, *tmX, a);
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;

@@ -16,7 +16,8 @@ struct ProfScope {
     ~ProfScope() { prof_end(kind, s); }
 };
 
-// ------------------------------------------------------------------ tensor-core GEMM (gemm_tcgen05.cu)
+// ------------------------------------------------------------------ tensor-core GEMM with split-K partial sums in global memory (gemm_tcgen05.cu)
+// The exported building block tasc_gemm_bf16 / tasc_gemm_bf16_static; the forward uses gemm_fused.cu.
 // Computes partial sums P[s][m][n] = sum over the k-range of split s of X[m][k] * W[n][k]
 // (bf16 inputs, float32 accumulation in TMEM).  Consumers add the `splits` slices in order.
 struct GemmPlan {
@@ -36,11 +37,8 @@ inline size_t gemm_partial_bytes(const GemmPlan& p, int M, int N) { return (size
 // rows x cols bf16 row-major matrix, box = {64 cols, box_rows}, 128-byte swizzle.
 tasc_status encode_tmap_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
-// argmax != null: LM-head mode (splits must be 1): per token row an atomic max of (value, id) is kept in
-// argmax[m] instead of writing partials; `logits` (nullable) additionally receives the full rows.
 tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, float* partials, int M, int N, int K,
-                             const GemmPlan& plan, unsigned long long* argmax, float* logits, int* status,
-                             cudaStream_t stream);
+                             const GemmPlan& plan, int* status, cudaStream_t stream);
 tasc_status gemm_set_attributes();
 
 // ------------------------------------------------------------------ fused projection GEMMs (gemm_fused.cu)
@@ -101,11 +99,10 @@ struct RowPlan {              // per-step row bookkeeping, all device pointers i
 // Rows of a verify step: [last committed token, drafts] at positions len-1 ..; skipped when len >= stop_len.
 void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len,
                         const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
-                        unsigned int* counters, int n_counters, cudaStream_t stream);
+                        cudaStream_t stream);
 // Rows of prefill chunk c: committed tokens c*R .. c*R+R-1, limited to positions <= len-2.
 void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
-                         int chunk, int vocab, int* status, unsigned int* counters, int n_counters, cudaStream_t stream);
-// (both also zero `counters`, the attention merge tickets, when given)
+                         int chunk, int vocab, int* status, cudaStream_t stream);
 
 // bf16 model: x[m] = embed[tok]; a_out = (hi, lo) of x * gain; ssq[m][0] = sum x^2, other slots 0; argmax[m] = 0.
 void launch_embed_scaled(const __nv_bfloat16* embed, const int* row_tok, const float* gain, float* x, __nv_bfloat16* a_out,

@@ -19,10 +19,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 __global__ void rows_verify_kernel(RowPlan rp, const int32_t* tokens, int64_t stride, const int32_t* len,
-                                   const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
-                                   unsigned int* counters, int n_counters) {
+                                   const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    for (int c = i; c < n_counters; c += gridDim.x * blockDim.x) counters[c] = 0u;
     if (i >= B * R) return;
     const int b = i / R, r = i % R;
     const int L = len[b];
@@ -42,9 +40,8 @@ __global__ void rows_verify_kernel(RowPlan rp, const int32_t* tokens, int64_t st
 }
 
 __global__ void rows_prefill_kernel(RowPlan rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
-                                    int chunk, int vocab, int* status, unsigned int* counters, int n_counters) {
+                                    int chunk, int vocab, int* status) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    for (int c = i; c < n_counters; c += gridDim.x * blockDim.x) counters[c] = 0u;
     if (i >= B * R) return;
     const int b = i / R, r = i % R;
     const int L = len[b];
@@ -293,16 +290,14 @@ __global__ void min_generated_kernel(const int32_t* len, const int32_t* prompt_l
 
 void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len,
                         const int32_t* stop_len, const int32_t* drafts, int B, int R, int vocab, int* status,
-                        unsigned int* counters, int n_counters, cudaStream_t stream) {
+                        cudaStream_t stream) {
     ProfScope ps(K_ROWS, stream);
-    rows_verify_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, stop_len, drafts, B, R, vocab, status,
-                                                                counters, n_counters);
+    rows_verify_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, stop_len, drafts, B, R, vocab, status);
 }
 void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
-                         int chunk, int vocab, int* status, unsigned int* counters, int n_counters, cudaStream_t stream) {
+                         int chunk, int vocab, int* status, cudaStream_t stream) {
     ProfScope ps(K_ROWS, stream);
-    rows_prefill_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, B, R, chunk, vocab, status,
-                                                                 counters, n_counters);
+    rows_prefill_kernel<<<(B * R + 127) / 128, 128, 0, stream>>>(rp, tokens, stride, len, B, R, chunk, vocab, status);
 }
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
@@ -391,6 +386,5 @@ void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, 
                                             cudaStream_t);                                                               \
     template void launch_silu_mul<T>(const float*, int, T*, int, int, int, cudaStream_t);
 TASC_INSTANTIATE(float)
-TASC_INSTANTIATE(__nv_bfloat16)
 
 }  // namespace tasc

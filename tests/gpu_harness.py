@@ -34,11 +34,15 @@ class Setup:
     drafter: object = None
 
 
-def make_setup(cfg, *, n_docs=None, gain_jitter=0.0, build_drafter=True, oracle_ngrams=True) -> Setup:
+def make_setup(cfg, *, n_docs=None, gain_jitter=0.0, build_drafter=True, oracle_ngrams=True, host_w=None,
+               corpus_tokens=None) -> Setup:
+    """``host_w`` / ``corpus_tokens`` = (tokens, offsets) replace the configuration's generated weights / corpus
+    (cfg.model must then describe the given weights)."""
     b = need_gpu()
     shape = cfg.model
-    host_w = W.make_weights(shape, cfg.seed_weights, gain_jitter=gain_jitter)
-    tokens, offsets = corpus.make_corpus(cfg, n_docs=n_docs)
+    if host_w is None:
+        host_w = W.make_weights(shape, cfg.seed_weights, gain_jitter=gain_jitter)
+    tokens, offsets = corpus.make_corpus(cfg, n_docs=n_docs) if corpus_tokens is None else corpus_tokens
     ng = D.build_corpus_ngrams_sorted(tokens, offsets, cfg.n_max, cfg.p_min, shape.vocab) if oracle_ngrams else None
     s = Setup(cfg, shape, host_w, OracleModel(shape, host_w, np.float32), ng, tokens, offsets)
     dev_w = b.weights_to_device(host_w, shape.dtype)

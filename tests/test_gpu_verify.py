@@ -157,3 +157,50 @@ def test_config2_lockstep_short():
     s = make_setup(cfg, n_docs=20000)
     prompts = corpus.make_prompts(cfg, 2)
     check(lockstep(s, prompts, 18, 8, **BF16_TOL))
+
+
+@pytest.mark.gpu
+def test_config3_expanded_vocabulary_lockstep():
+    """Configuration 3: 8,192 merged n-gram tokens on top of the 0.5B vocabulary (V = 160,128), embedding rows
+    initialised as constituent means, corpus and prompts re-tokenised by greedy longest match.  Two layers and a
+    3,000-document corpus keep the oracle quick; the LM head / argmax and the drafter run at the full vocabulary."""
+    from dataclasses import replace
+    from workload import vocab_expand as VE, weights as W
+    cfg3 = configs.get(3)
+    base = cfg3.model.vocab
+    small = configs.shrunk(cfg3, n_layers=2, n_docs=3000)
+    toks, offs = corpus.make_corpus(small)
+    merges = VE.select_merges(toks, offs, cfg3.n_merged_tokens, n_max=4, vocab=base)
+    assert len(merges) == cfg3.n_merged_tokens
+    toks2, offs2 = VE.retokenize(toks, offs, merges, vocab=base)
+    host_w = VE.expand_weights(W.make_weights(small.model, small.seed_weights), merges)
+    cfg = replace(small, model=replace(small.model, vocab=base + len(merges)))
+    s = make_setup(cfg, host_w=host_w, corpus_tokens=(toks2, offs2))
+    raw = corpus.make_prompts(small, 2)
+    re = [VE.retokenize(raw[i], np.array([0, raw.shape[1]]), merges, vocab=base)[0] for i in range(2)]
+    P = min(len(r) for r in re)
+    prompts = np.stack([r[:P] for r in re]).astype(np.int32)
+    assert prompts.max() >= base                      # merged tokens do occur in the prompts
+    check(lockstep(s, prompts, 12, cfg.k, **BF16_TOL))
+
+
+@pytest.mark.gpu
+def test_config4_shape_long_context_lockstep():
+    """Configuration 4's geometry (d_model 1536, 12 query / 2 KV heads of 128, d_ff 8960, n_max 5, k 6, prompts of
+    1,024 tokens) with two layers and a 32k vocabulary: 128-wide heads, a context long enough for the key range of a
+    (sequence, KV head) to be split over a cluster, and prefill chunks of 96 query rows per KV head."""
+    cfg = configs.shrunk(configs.get(4), n_layers=2, vocab=32768, n_docs=20000)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 2)
+    check(lockstep(s, prompts, 14, cfg.k, **BF16_TOL))
+
+
+@pytest.mark.gpu
+def test_config2_batch32_k3_and_k8_one_step():
+    """Batch 32 of configuration 2's geometry at k = 3 (M = 128 rows, one token tile) and k = 8 (M = 288 rows, three
+    token tiles of 96), two layers."""
+    cfg = configs.shrunk(configs.get(2), n_layers=2, vocab=32768, n_docs=5000)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 32, prompt_len=80)
+    for k in (3, 8):
+        check(lockstep(s, prompts, k + 1, k, **BF16_TOL))
