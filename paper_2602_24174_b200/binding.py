@@ -135,7 +135,7 @@ class Drafter:
         self._h, self.n_max = handle, n_max
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and lib is not None:      # lib is None while the interpreter shuts down
             lib.tasc_drafter_destroy(self._h)
             self._h = None
 
@@ -207,7 +207,7 @@ class Model:
         self._h = h
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and lib is not None:
             lib.tasc_model_destroy(self._h)
             self._h = None
 

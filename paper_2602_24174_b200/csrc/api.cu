@@ -115,11 +115,21 @@ KvView layer_kv(const tasc_model* m, const tasc_kv* kv, int layer) {
     return KvView{base, base + per};
 }
 
+// Where the rows of a forward come from: a verify step (chunk < 0: last committed token + drafts) or prefill chunk `chunk`.
+struct RowSource {
+    const tasc_seqs* seqs;
+    const int32_t* drafts;
+    int chunk;
+};
+
 // float32 model (the tiny configuration): one launch per stage, float32 SIMT kernels.
-tasc_status forward_f32(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
-                        cudaStream_t s) {
+tasc_status forward_f32(const tasc_model* m, const tasc_kv* kv, const Workspace& w, const RowSource& src, int B, int R, bool lm_head,
+                        float* logits, cudaStream_t s) {
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
+    const tasc_seqs* sq = src.seqs;
+    if (src.chunk < 0) launch_rows_verify(w.rp, sq->tokens, sq->stride, sq->len, sq->stop_len, src.drafts, B, R, d.vocab, w.status, s);
+    else launch_rows_prefill(w.rp, sq->tokens, sq->stride, sq->len, B, R, src.chunk, d.vocab, w.status, s);
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
     const int att_splits = attention_splits(B, d.n_kv_heads, max_ctx);
     float* h = static_cast<float*>(w.h);
@@ -157,8 +167,8 @@ tasc_status forward_f32(const tasc_model* m, const tasc_kv* kv, const Workspace&
 
 // bf16 models: five launches per layer (QKV+RoPE+KV append, attention, O+residual, gate/up+SiLU*mul, down+residual),
 // each with programmatic stream serialisation; see gemm_fused.cu and attention_mma.cu.
-tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
-                         cudaStream_t s) {
+tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace& w, const RowSource& src, int B, int R,
+                         bool lm_head, float* logits, cudaStream_t s) {
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
@@ -185,8 +195,9 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     base.eps = d.rms_eps;
     base.status = w.status;
 
-    launch_embed_scaled(static_cast<const __nv_bfloat16*>(m->embed), w.rp.row_tok, m->attn_norm[0], w.x, h, w.ssq, w.ssq_slots,
-                        lm_head ? w.argmax : nullptr, M, d.d_model, TB, s);
+    launch_rows_embed(w.rp, src.seqs->tokens, src.seqs->stride, src.seqs->len, src.seqs->stop_len, src.drafts, B, R, src.chunk,
+                      d.vocab, w.status, static_cast<const __nv_bfloat16*>(m->embed), m->attn_norm[0], w.x, h, w.ssq, w.ssq_slots,
+                      lm_head ? w.argmax : nullptr, d.d_model, TB, s);
     for (int l = 0; l < d.n_layers; ++l) {
         const KvView kvl = layer_kv(m, kv, l);
         FusedArgs a = base;
@@ -225,10 +236,10 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     return TASC_OK;
 }
 
-tasc_status forward_any(const tasc_model* m, const tasc_kv* kv, const Workspace& w, int B, int R, bool lm_head, float* logits,
-                        cudaStream_t s) {
-    return m->desc.dtype == TASC_F32 ? forward_f32(m, kv, w, B, R, lm_head, logits, s)
-                                     : forward_bf16(m, kv, w, B, R, lm_head, logits, s);
+tasc_status forward_any(const tasc_model* m, const tasc_kv* kv, const Workspace& w, const RowSource& src, int B, int R,
+                        bool lm_head, float* logits, cudaStream_t s) {
+    return m->desc.dtype == TASC_F32 ? forward_f32(m, kv, w, src, B, R, lm_head, logits, s)
+                                     : forward_bf16(m, kv, w, src, B, R, lm_head, logits, s);
 }
 
 bool check_common(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, int B, void* ws, size_t ws_bytes) {
@@ -243,8 +254,7 @@ tasc_status verify_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_se
                            const int32_t* drafts, int B, int k, const int32_t* forced, int32_t* n_accepted,
                            int32_t* next_token, int32_t* target_tokens, float* logits, cudaStream_t s) {
     const int R = k + 1;
-    launch_rows_verify(w.rp, seqs->tokens, seqs->stride, seqs->len, seqs->stop_len, drafts, B, R, m->desc.vocab, w.status, s);
-    tasc_status st = forward_any(m, kv, w, B, R, true, logits, s);
+    tasc_status st = forward_any(m, kv, w, RowSource{seqs, drafts, -1}, B, R, true, logits, s);
     if (st != TASC_OK) return st;
     launch_accept(w.argmax, w.rp, drafts, forced, seqs->tokens, seqs->stride, seqs->len, B, R, n_accepted, next_token,
                   target_tokens, w.hist, s);
@@ -257,8 +267,7 @@ tasc_status prefill_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_s
     const int R = TASC_MAX_ROWS;
     const int chunks = (std::max(max_len - 1, 0) + R - 1) / R;
     for (int c = 0; c < chunks; ++c) {
-        launch_rows_prefill(w.rp, seqs->tokens, seqs->stride, seqs->len, B, R, c, m->desc.vocab, w.status, s);
-        tasc_status st = forward_any(m, kv, w, B, R, false, nullptr, s);
+        tasc_status st = forward_any(m, kv, w, RowSource{seqs, nullptr, c}, B, R, false, nullptr, s);
         if (st != TASC_OK) return st;
     }
     return TASC_OK;

@@ -512,18 +512,18 @@ int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
 
 // Key-range splits per (sequence, KV head), 1..8 (a cluster), from a small cost model in microseconds: a CTA
 // needs about 1.5 us to start plus one tile time per iteration (its warp groups take `ng` tiles per iteration),
-// all CTAs run in waves of about two per SM, and splitting adds the cluster exchange and merge (about 3 us).
+// all CTAs run in waves of about two per SM, and splitting adds the cluster exchange and merge (about 4.5 us).
 int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx) {
     const int n_tiles = (max_ctx + TKEYS - 1) / TKEYS;
     const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;
     const int ng = (hd < 128 && nw / n_slabs >= 2) ? 2 : 1;
-    const float t_tile = hd >= 128 ? 0.9f : (hd >= 64 ? 0.45f : 0.3f);
+    const float t_tile = hd >= 128 ? 0.9f : (hd >= 64 ? 0.4f : 0.3f);
     int best = 1;
     float best_cost = 1e30f;
     for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
         const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
         const int waves = (B * n_kv * s + 295) / 296;
-        const float cost = waves * (1.5f + iters * t_tile) + (s > 1 ? 3.0f : 0.f);
+        const float cost = waves * (1.5f + iters * t_tile) + (s > 1 ? 4.5f : 0.f);
         if (cost < best_cost - 1e-6f) { best_cost = cost; best = s; }
     }
     return best;

@@ -8,8 +8,8 @@
 // plus a flat successor array of (next, count).  Slot placement depends on thread timing, results do
 // not: lookups return the same sets, and the export sorts canonically.
 //
-// Draft (every step): one CTA per sequence.  For each of the k drafts: warp-cooperative back-off probe
-// of the context tables (32 slots per probe round), a scan of the sequence's committed tokens for the
+// Draft (every step): one CTA per sequence.  For each of the k drafts: warp-cooperative probes of the
+// context tables of all orders at once (one warp per order, 32 slots per probe round; longest hit wins), a scan of the sequence's committed tokens for the
 // longest matching suffix with its successor counts collected in a shared-memory hash, and the argmax
 // of  lambda_num * c_corp(x) * T_prompt + (lambda_den - lambda_num) * c_prompt(x) * T_corp  in 64-bit
 // integers with the smallest token id winning ties.
@@ -253,8 +253,9 @@ draft_kernel(const DeviceTables dt, const int32_t* __restrict__ tokens, int64_t 
     uint32_t* h_cnt = reinterpret_cast<uint32_t*>(dsm + hs_mask + 1);   // [hs] count, bit 31 = seen in the corpus list
     __shared__ Best red[DRAFT_THREADS / 32];
     __shared__ int s_suffix[TASC_MAX_ORDER];     // last n_max tokens of the query, newest last
-    __shared__ int s_nstar, s_tprompt, s_found_n;
-    __shared__ CtxVal s_val;
+    __shared__ int s_nstar, s_tprompt;
+    __shared__ int s_hit[TASC_MAX_ORDER];        // order n = index + 1 has a surviving context for the current suffix
+    __shared__ CtxVal s_vals[TASC_MAX_ORDER];
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -273,18 +274,19 @@ draft_kernel(const DeviceTables dt, const int32_t* __restrict__ tokens, int64_t 
     for (int j = 0; j < k; ++j) {
         const int Lq = L + j;                      // query length so far
         const int n_avail = Lq < n_max ? Lq : n_max;
-        // ---------------------------------------------------------------- p_corp: back-off probe (warp 0)
-        if (warp == 0) {
-            int found = 0;
+        // ---------------------------------------------------------------- p_corp: all orders are probed at once, one warp
+        // per order (warp w looks up the last w + 1 tokens); the longest order that matched wins the back-off
+        if (tid == 0) { s_nstar = 0; s_tprompt = 0; }
+        if (warp < TASC_MAX_ORDER) {
+            const int n = warp + 1;
+            bool hit = false;
             CtxVal val = {0ull, 0u, 0u};
-            if (use_corp) {
-                for (int n = n_avail; n >= 1 && !found; --n) {
-                    Key key = key_make(n);
-                    for (int i = 0; i < n; ++i) key_put(key, i, (uint32_t)s_suffix[n_max - n + i]);
-                    if (warp_lookup(dt.t[n], key, val)) found = n;
-                }
+            if (use_corp && n <= n_avail) {
+                Key key = key_make(n);
+                for (int i = 0; i < n; ++i) key_put(key, i, (uint32_t)s_suffix[n_max - n + i]);
+                hit = warp_lookup(dt.t[n], key, val);
             }
-            if (tid == 0) { s_found_n = found; s_val = val; s_nstar = 0; s_tprompt = 0; }
+            if ((tid & 31) == 0) { s_hit[warp] = hit ? 1 : 0; s_vals[warp] = val; }
         }
         // ---------------------------------------------------------------- p_prompt: longest suffix match in the committed tokens
         if (use_prompt)
@@ -318,8 +320,10 @@ draft_kernel(const DeviceTables dt, const int32_t* __restrict__ tokens, int64_t 
             }
             __syncthreads();
         }
-        const int found_n = s_found_n;
-        const CtxVal cv = s_val;
+        int found_n = 0;
+        for (int n = n_max; n >= 1 && !found_n; --n)
+            if (s_hit[n - 1]) found_n = n;
+        const CtxVal cv = s_vals[found_n > 0 ? found_n - 1 : 0];
         const unsigned long long t_corp = cv.total;
         const unsigned long long t_prompt = (unsigned long long)s_tprompt;
         const bool has_corp = found_n > 0, has_prompt = t_prompt > 0;

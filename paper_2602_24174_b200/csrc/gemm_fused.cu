@@ -92,7 +92,9 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int BN = a.BN, stages = a.stages, TB = a.TB;
     const uint32_t b_stage_bytes = (uint32_t)BN * BK * 2;
     const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
-    float* xch = reinterpret_cast<float*>(smem + (size_t)stages * stage_bytes);          // [TB][128] this CTA's partial tile
+    // [TB][128] this CTA's partial tile; behind the ring, except for the LM head, which has no cluster exchange
+    // and parks it in the ring once its MMAs are done
+    float* xch = reinterpret_cast<float*>(EPI == EPI_LM ? smem : smem + (size_t)stages * stage_bytes);
     float* fin = reinterpret_cast<float*>(smem);                                          // [per][128] reduced columns (the ring is idle by then)
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + a.data_bytes);
     const uint32_t bar_full = smem_u32(bars);
@@ -596,24 +598,26 @@ FusedPlan plan_fused(int M, int N, int K, int epi) {
     const int stage_bytes = A_STAGE_BYTES + p.BN * BK * 2;
     int ncols = 32;
     while (ncols < p.BN) ncols <<= 1;
-    const int xch_bytes = p.TB * BM * 4;                        // the CTA's partial tile for the split-K exchange, not aliased with the ring
+    // the CTA's partial tile for the split-K exchange, not aliased with the ring (the LM head reuses the ring)
+    const int xch_bytes = epi == EPI_LM ? 0 : p.TB * BM * 4;
     for (;; --S) {
         p.S = S;
         const int kb_per = (p.num_kb + S - 1) / S;
         // A CTA's streaming rate is its bytes in flight over the memory latency.  A grid of one wave (at most
-        // one CTA per SM anyway) gets a ring of up to 200 KB; a grid of several waves with narrow tiles keeps
-        // about 100 KB per CTA so that two CTAs share an SM and cover each other's start-up and epilogue.
+        // one CTA per SM anyway) gets a ring of up to 200 KB; a grid of several waves keeps about 100 KB per
+        // CTA so that two CTAs share an SM and cover each other's start-up and epilogue.
         const bool one_wave = tiles * S <= 148;
-        const int budget = ((ncols <= 128 && !one_wave) ? 100 * 1024 : 216 * 1024) - xch_bytes;
+        const int budget = ((ncols <= 128 || epi == EPI_LM) && !one_wave ? 108 * 1024 : 216 * 1024) - xch_bytes;
         int st = budget / stage_bytes;
         st = std::max(2, std::min(st, 8));
         st = std::min(st, std::max(2, kb_per));
         p.stages = st;
-        p.data_bytes = st * stage_bytes + xch_bytes;
+        p.data_bytes = std::max(st * stage_bytes, p.TB * BM * 4) + xch_bytes;
         int smem = 1024 + p.data_bytes + (2 * st + 2) * 8 + 128 * 4;
         // TMEM columns held by co-resident CTAs must never exceed 512, or CTAs of different clusters can
         // block each other's allocation while waiting at a cluster barrier: shared memory limits residency.
-        smem = std::max(smem, ncols * 454 + 1);
+        // (The LM head has no cluster barrier to wait at; two of its CTAs with 256 columns each share an SM.)
+        if (epi != EPI_LM) smem = std::max(smem, ncols * 454 + 1);
         p.smem_bytes = std::min(smem, MAX_DYN_SMEM);
         if (S == 1) break;
         // All clusters of the grid should be resident at once: a second, nearly empty wave doubles the

@@ -104,13 +104,16 @@ void launch_rows_verify(const RowPlan& rp, const int32_t* tokens, int64_t stride
 void launch_rows_prefill(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, int B, int R,
                          int chunk, int vocab, int* status, cudaStream_t stream);
 
-// bf16 model: x[m] = embed[tok]; a_out = (hi, lo) of x * gain; ssq[m][0] = sum x^2, other slots 0; argmax[m] = 0.
-void launch_embed_scaled(const __nv_bfloat16* embed, const int* row_tok, const float* gain, float* x, __nv_bfloat16* a_out,
-                         float* ssq, int ssq_slots, unsigned long long* argmax, int M, int d, int TB, cudaStream_t stream);
-
+// float32 model: x[m] = embed[tok]; h[m] = RMSNorm(x[m]) * gain
 template <typename T>
 void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, float eps, float* x, T* h, int M, int d,
                        int TB, cudaStream_t stream);
+// bf16 model, first launch of a forward: row plan (chunk < 0: verify step, else prefill chunk) + embedding:
+// x[m] = embed[tok]; a_out = (hi, lo) of x * gain; ssq[m][0] = sum x^2, other slots 0; argmax[m] = 0 (if given).
+void launch_rows_embed(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, const int32_t* stop_len,
+                       const int32_t* drafts, int B, int R, int chunk, int vocab, int* status, const __nv_bfloat16* embed,
+                       const float* gain, float* x, __nv_bfloat16* a_out, float* ssq, int ssq_slots, unsigned long long* argmax,
+                       int d, int TB, cudaStream_t stream);
 // x += sum_s P[s]; h = RMSNorm(x) * gain  (gain == null: only the residual update)
 template <typename T>
 void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,

@@ -82,14 +82,50 @@ embed_norm_kernel(const T* __restrict__ embed, const int* __restrict__ row_tok, 
         ActStore<T>::put(h, m, j, d, TB, x[(size_t)m * d + j] * inv * gain[j]);
 }
 
-// bf16 model: the RMS factor is applied by the consumer GEMM, so the row leaves here as x * gain plus its sum of squares
+// bf16 model, first launch of a forward: the row plan of a verify step (chunk < 0: rows = [last committed token,
+// drafts] at positions len-1 ..; skipped when len >= stop_len) or of prefill chunk `chunk` (committed tokens
+// chunk*R .. limited to positions <= len-2), and the embedding of every row.  The RMS factor is applied by the
+// consumer GEMM, so the row leaves here as x * gain (hi, lo) plus its sum of squares.
 __global__ void __launch_bounds__(128)
-embed_scaled_kernel(const __nv_bfloat16* __restrict__ embed, const int* __restrict__ row_tok, const float* __restrict__ gain,
-                    float* __restrict__ x, __nv_bfloat16* __restrict__ a_out, float* __restrict__ ssq, int ssq_slots,
-                    unsigned long long* argmax, int d, int TB) {
+rows_embed_kernel(RowPlan rp, const int32_t* __restrict__ tokens, int64_t stride, const int32_t* __restrict__ len,
+                  const int32_t* __restrict__ stop_len, const int32_t* __restrict__ drafts, int R, int chunk, int vocab,
+                  int* status, const __nv_bfloat16* __restrict__ embed, const float* __restrict__ gain, float* __restrict__ x,
+                  __nv_bfloat16* __restrict__ a_out, float* __restrict__ ssq, int ssq_slots, unsigned long long* argmax, int d,
+                  int TB) {
     __shared__ float red[4];
+    __shared__ int s_tok;
     const int m = blockIdx.x;
-    const __nv_bfloat16* e = embed + (size_t)row_tok[m] * d;
+    if (threadIdx.x == 0) {
+        const int b = m / R, r = m % R;
+        const int L = len[b];
+        const bool len_ok = L >= 1 && L <= stride;
+        if (!len_ok) set_status(status, TASC_EINVAL);
+        int tok = 0, pos = -1, pos0 = 0, rows = 0;
+        if (chunk < 0) {
+            const bool active = len_ok && !(stop_len && L >= stop_len[b]);
+            if (active) {
+                tok = r == 0 ? tokens[(int64_t)b * stride + L - 1] : drafts[b * (R - 1) + r - 1];
+                pos = L - 1 + r;
+                pos0 = L - 1;
+                rows = R;
+            }
+        } else {
+            pos0 = chunk * R;
+            rows = len_ok ? L - 1 - pos0 : 0;
+            rows = rows < 0 ? 0 : (rows > R ? R : rows);
+            if (r < rows) {
+                tok = tokens[(int64_t)b * stride + pos0 + r];
+                pos = pos0 + r;
+            }
+        }
+        if (tok < 0 || tok >= vocab) { set_status(status, TASC_EINVAL); tok = 0; }
+        rp.row_tok[m] = tok;
+        rp.row_pos[m] = pos;
+        if (r == 0) { rp.seq_pos0[b] = pos0; rp.seq_rows[b] = rows; }
+        s_tok = tok;
+    }
+    __syncthreads();
+    const __nv_bfloat16* e = embed + (size_t)s_tok * d;
     float ss = 0.f;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
         const float v = __bfloat162float(e[j]);
@@ -305,10 +341,13 @@ void launch_embed_norm(const T* embed, const int* row_tok, const float* gain, fl
     ProfScope ps(K_EMBED, stream);
     embed_norm_kernel<T><<<M, 128, 0, stream>>>(embed, row_tok, gain, eps, x, h, d, TB);
 }
-void launch_embed_scaled(const __nv_bfloat16* embed, const int* row_tok, const float* gain, float* x, __nv_bfloat16* a_out,
-                         float* ssq, int ssq_slots, unsigned long long* argmax, int M, int d, int TB, cudaStream_t stream) {
+void launch_rows_embed(const RowPlan& rp, const int32_t* tokens, int64_t stride, const int32_t* len, const int32_t* stop_len,
+                       const int32_t* drafts, int B, int R, int chunk, int vocab, int* status, const __nv_bfloat16* embed,
+                       const float* gain, float* x, __nv_bfloat16* a_out, float* ssq, int ssq_slots, unsigned long long* argmax,
+                       int d, int TB, cudaStream_t stream) {
     ProfScope ps(K_EMBED, stream);
-    embed_scaled_kernel<<<M, 128, 0, stream>>>(embed, row_tok, gain, x, a_out, ssq, ssq_slots, argmax, d, TB);
+    rows_embed_kernel<<<B * R, 128, 0, stream>>>(rp, tokens, stride, len, stop_len, drafts, R, chunk, vocab, status, embed, gain,
+                                                 x, a_out, ssq, ssq_slots, argmax, d, TB);
 }
 template <typename T>
 void launch_residual_norm(const float* partials, int splits, float* x, const float* gain, float eps, T* h, int M, int d,
