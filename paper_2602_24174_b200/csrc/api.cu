@@ -172,7 +172,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
-    const int att_splits = attention_mma_splits(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * R, max_ctx);
+    const AttnPlan att_plan = plan_attention_mma(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * R, max_ctx);
     const int TB = gemm_token_tile(M, true);
     const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
     CUtensorMap tm_h, tm_o, tm_act;
@@ -210,7 +210,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
 
         st = launch_attention_mma(w.q, static_cast<const __nv_bfloat16*>(kvl.k), static_cast<const __nv_bfloat16*>(kvl.v),
                                   kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, B, R,
-                                  d.n_q_heads, d.n_kv_heads, d.head_dim, att_splits, s);
+                                  d.n_q_heads, d.n_kv_heads, d.head_dim, att_plan, s);
         if (st != TASC_OK) return st;
 
         a = base;

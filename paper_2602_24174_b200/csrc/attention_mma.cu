@@ -19,6 +19,10 @@
 // writes it as (hi, lo) bf16 in the layout the O-projection GEMM loads.  Nothing goes through global memory.
 #include "kernels.h"
 
+#include <algorithm>
+#include <map>
+#include <mutex>
+
 namespace tasc {
 
 namespace {
@@ -36,7 +40,7 @@ struct AttnArgs {
     const int* seq_rows;
     __nv_bfloat16* out;                // (hi, lo) activation buffer, row length n_q * hd
     int TB;
-    int R, n_q, n_kv, splits;
+    int R, n_q, n_kv, splits, stages;
     float scale_log2e;
 };
 
@@ -77,9 +81,23 @@ __device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32
     lo = (uint32_t)__bfloat16_as_ushort(lx) | ((uint32_t)__bfloat16_as_ushort(ly) << 16);
 }
 
-// Ring depth of the K/V tile pipeline.  A CTA streams its key range alone, so the bytes it keeps in flight
-// (ring depth x 8-32 KB per tile) over the memory latency are its bandwidth: 100-190 KB of tiles per CTA.
-template <int HD, int NW> struct Ring { static constexpr int STAGES = HD >= 128 ? (NW > 4 ? 4 : 5) : 8; };
+// Largest ring depth of the K/V tile pipeline (the host picks 2..max per launch).  A CTA streams its key range
+// alone, so the bytes it keeps in flight (ring depth x 8-32 KB per tile) over the memory latency are its
+// bandwidth; a shallower ring lets two CTAs share an SM when many (sequence, KV head) pairs are in flight.
+template <int HD, int NW> struct Ring { static constexpr int MAX_STAGES = HD >= 128 ? (NW > 4 ? 4 : 5) : 8; };
+
+__device__ __forceinline__ void cp_async_wait_dyn(int n) {      // wait until at most n groups are pending
+    switch (n) {
+        case 0: cp_async_wait<0>(); break;
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        case 6: cp_async_wait<6>(); break;
+        default: cp_async_wait<7>(); break;
+    }
+}
 
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32)
@@ -88,7 +106,7 @@ attn_mma_kernel(const AttnArgs a) {
     constexpr int CH = HD / 8;                   // 16-byte chunks per row
     constexpr int THREADS = NW * 32;
     constexpr int TILE_BYTES = TKEYS * HD * 2;
-    constexpr int STAGES = Ring<HD, NW>::STAGES;
+    const int STAGES = a.stages;                 // ring depth of this launch, 2 .. Ring<HD, NW>::MAX_STAGES
     extern __shared__ __align__(128) uint8_t sm[];
     uint8_t* Qh = sm;
     uint8_t* Ql = Qh + GP * HD * 2;
@@ -243,7 +261,7 @@ attn_mma_kernel(const AttnArgs a) {
     for (int sup = 0; sup < n_super; ++sup) {
         if (sup + super_stages - 1 < n_super) load_super(sup + super_stages - 1);
         else cp_async_commit();
-        if (ng == 1) cp_async_wait<STAGES - 1>(); else cp_async_wait<STAGES / 2 - 1>();   // iteration `sup` has landed
+        cp_async_wait_dyn(super_stages - 1);                      // iteration `sup` has landed
         __syncthreads();
 #ifdef TASC_TIMELINE
         if (sup == 0) log_at_exit.td = global_ns();
@@ -471,10 +489,12 @@ attn_mma_kernel(const AttnArgs a) {
     cluster_wait();
 }
 
+inline size_t attn_smem_bytes(int hd, int gp, int stages) {
+    return (size_t)2 * gp * hd * 2 + (size_t)2 * stages * TKEYS * hd * 2;
+}
+
 template <int HD, int NW>
-tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
-    constexpr int GP = NW * 16;
-    const size_t smem = (size_t)2 * GP * HD * 2 + (size_t)2 * Ring<HD, NW>::STAGES * TKEYS * HD * 2;
+tasc_status prepare_inst() {
     static bool done[64] = {false};
     int dev = 0;
     TASC_CUDA_TRY(cudaGetDevice(&dev));
@@ -483,6 +503,52 @@ tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
         TASC_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<HD, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         done[dev] = true;
     }
+    return TASC_OK;
+}
+
+// Clusters of `splits` CTAs (ring depth `stages`) the device holds at once; 0 if the query fails.
+template <int HD, int NW>
+int fit_inst(int splits, int stages) {
+    if (prepare_inst<HD, NW>() != TASC_OK) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)splits, 1, 1);
+    cfg.blockDim = dim3(NW * 32, 1, 1);
+    cfg.dynamicSmemBytes = attn_smem_bytes(HD, NW * 16, stages);
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)splits;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, attn_mma_kernel<HD, NW>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return n;
+}
+
+int fit_any(int hd, int nw, int splits, int stages) {
+    static std::mutex mu;
+    static std::map<long long, int> cache;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    const long long key = ((((long long)dev * 256 + hd) * 16 + nw) * 16 + splits) * 16 + stages;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    int n = 0;
+    if (nw == 4) n = hd == 32 ? fit_inst<32, 4>(splits, stages) : hd == 64 ? fit_inst<64, 4>(splits, stages) : fit_inst<128, 4>(splits, stages);
+    else n = hd == 32 ? fit_inst<32, 8>(splits, stages) : hd == 64 ? fit_inst<64, 8>(splits, stages) : fit_inst<128, 8>(splits, stages);
+    cache[key] = n;
+    return n;
+}
+
+template <int HD, int NW>
+tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
+    constexpr int GP = NW * 16;
+    if (a.stages < 2 || a.stages > Ring<HD, NW>::MAX_STAGES) return TASC_EINVAL;
+    const size_t smem = attn_smem_bytes(HD, GP, a.stages);
+    tasc_status pst = prepare_inst<HD, NW>();
+    if (pst != TASC_OK) return pst;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)a.splits, (unsigned)a.n_kv, (unsigned)B);
     cfg.blockDim = dim3(NW * 32, 1, 1);
@@ -510,21 +576,31 @@ tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
 
 int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
 
-// Key-range splits per (sequence, KV head), 1..8 (a cluster), from a small cost model in microseconds: a CTA
-// needs about 1.5 us to start plus one tile time per iteration (its warp groups take `ng` tiles per iteration),
-// all CTAs run in waves of about two per SM, and splitting adds the cluster exchange and merge (about 4.5 us).
-int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx) {
+// Key-range splits per (sequence, KV head) (1..8, the CTAs of a cluster) and ring depth, from a small cost model
+// in microseconds: a CTA needs about 1.5 us to start plus one tile time per iteration (its warp groups take `ng`
+// tiles per iteration; a shallow ring adds memory stalls), the clusters run in as many waves as the device's
+// cluster occupancy dictates (one straggling cluster costs a whole wave), and splitting adds the cluster
+// exchange and merge (about 4.5 us).
+AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx) {
     const int n_tiles = (max_ctx + TKEYS - 1) / TKEYS;
     const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;
-    const int ng = (hd < 128 && nw / n_slabs >= 2) ? 2 : 1;
+    const int max_stages = hd >= 128 ? (nw > 4 ? 4 : 5) : 8;
     const float t_tile = hd >= 128 ? 0.9f : (hd >= 64 ? 0.4f : 0.3f);
-    int best = 1;
+    AttnPlan best = {1, max_stages};
     float best_cost = 1e30f;
-    for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
-        const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
-        const int waves = (B * n_kv * s + 295) / 296;
-        const float cost = waves * (1.5f + iters * t_tile) + (s > 1 ? 4.5f : 0.f);
-        if (cost < best_cost - 1e-6f) { best_cost = cost; best = s; }
+    const int depths[2] = {max_stages, max_stages >= 8 ? 4 : 3};
+    for (int di = 0; di < 2; ++di) {
+        const int stages = depths[di];
+        const int ng = (stages >= 4 && nw / n_slabs >= 2) ? 2 : 1;
+        for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
+            int fit = fit_any(hd, nw, s, stages);
+            if (fit <= 0) fit = std::max(1, 148 / s);               // no device to ask: assume one CTA per SM
+            const int waves = (B * n_kv + fit - 1) / fit;
+            const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
+            const float stall = di == 0 ? 0.f : 0.25f * t_tile;      // a shallow ring hides less latency
+            const float cost = waves * (1.5f + iters * (t_tile + stall)) + (s > 1 ? 4.5f : 0.f);
+            if (cost < best_cost - 1e-6f) { best_cost = cost; best = AttnPlan{s, stages}; }
+        }
     }
     return best;
 }
@@ -532,7 +608,8 @@ int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx) {
 tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
                                  const int32_t* block_table, int max_pages, int page_size, long long n_pages,
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
-                                 int n_splits, cudaStream_t stream) {
+                                 const AttnPlan& plan, cudaStream_t stream) {
+    const int n_splits = plan.splits;
     const int G = (n_q / n_kv) * R;
     if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 8) return TASC_EINVAL;
     const int GP = attention_mma_row_pad(G);
@@ -541,7 +618,7 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
     a.max_pages = max_pages; a.page_size = page_size; a.n_pages = n_pages;
     a.seq_pos0 = rp.seq_pos0; a.seq_rows = rp.seq_rows;
     a.out = out; a.TB = TB;
-    a.R = R; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits;
+    a.R = R; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits; a.stages = plan.stages;
     a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
     if (GP == 64) {
         if (hd == 32) return launch_inst<32, 4>(a, B, stream);

@@ -157,11 +157,15 @@ int attention_splits(int B, int n_kv, int max_ctx);
 
 
 // ------------------------------------------------------------------ tensor-core attention for bf16 models (attention_mma.cu)
+struct AttnPlan {
+    int splits;      // key-range splits per (sequence, KV head) = cluster size, 1..8
+    int stages;      // depth of the K/V tile ring
+};
 // Same contract as launch_attention; the result goes to `out` as (hi, lo) bf16 rows; needs no scratch memory.
 tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
                                  const int32_t* block_table, int max_pages, int page_size, long long n_pages,
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
-                                 int n_splits, cudaStream_t stream);
-int attention_mma_splits(int B, int n_kv, int hd, int G, int max_ctx);     // 1..8 (the splits form a cluster)
+                                 const AttnPlan& plan, cudaStream_t stream);
+AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx);
 
 }  // namespace tasc
