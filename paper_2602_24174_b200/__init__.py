@@ -6,6 +6,9 @@ marshals torch CUDA tensors into it.  There is no CPU or PyTorch fallback: using
 without the built library raises ImportError.
 """
 
+# File name of the CUDA library inside this package that `binding` loads.
+LIBRARY_FILE = "libtasc.so"
+
 
 def __getattr__(name):
     if name == "binding":

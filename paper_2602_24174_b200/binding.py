@@ -13,7 +13,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtasc.so")
+from . import LIBRARY_FILE            # "libtasc.so"; timeline.py switches to the instrumented build of the same sources
+LIB_PATH = os.path.join(_HERE, LIBRARY_FILE)
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
