@@ -210,7 +210,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
 
         st = launch_attention_mma(w.q, static_cast<const __nv_bfloat16*>(kvl.k), static_cast<const __nv_bfloat16*>(kvl.v),
                                   kv->block_table, kv->max_pages_per_seq, d.page_size, kv->n_pages, w.rp, o, TB, B, R,
-                                  d.n_q_heads, d.n_kv_heads, d.head_dim, att_plan, s);
+                                  d.n_q_heads, d.n_kv_heads, d.head_dim, att_plan, w.status, s);
         if (st != TASC_OK) return st;
 
         a = base;

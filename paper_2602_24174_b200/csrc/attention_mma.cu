@@ -4,8 +4,9 @@
 // The kernel is bound by streaming K and V from HBM once; the tensor cores only have to keep up with
 // that stream, which a float32 SIMT formulation cannot do beyond a few sequences.  A CTA owns one
 // (sequence, KV head, key range): the key range of a sequence is split over several CTAs because the
-// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a 4-8 stage cp.async pipeline
-// (16-byte vectors, every page of a KV head is one contiguous run) into XOR-swizzled shared memory;
+// batch alone cannot fill 148 SMs.  K/V tiles of 64 keys arrive through a ring of 2-8 stages in swizzled shared
+// memory: one TMA box load per 16-token page (every page of a KV head is one contiguous run), issued by one
+// thread and signalled on an mbarrier; pools with another page size use 16-byte cp.async copies instead;
 // warp w computes the 16-row slab w of S = Q K^T and O += P V with mma.sync m16n8k16 (ldmatrix
 // fragments, V through ldmatrix.trans) and keeps an online softmax per row in registers.
 //
@@ -20,6 +21,7 @@
 #include "kernels.h"
 
 #include <algorithm>
+#include <cstring>
 #include <map>
 #include <mutex>
 
@@ -41,16 +43,21 @@ struct AttnArgs {
     __nv_bfloat16* out;                // (hi, lo) activation buffer, row length n_q * hd
     int TB;
     int R, n_q, n_kv, splits, stages;
+    int use_tma;                       // K/V tiles by TMA box loads (16-token pages); otherwise by cp.async
+    int* status;
     float scale_log2e;
 };
 
-// Byte offset of 16-byte chunk `chunk` of row `row` in a [rows][HD] bf16 tile; the XOR keeps the eight
-// rows of an ldmatrix phase on distinct banks.
-template <int HD>
+// Byte offset of 16-byte chunk `chunk` of row `row` in a 64-row bf16 tile (the Q tile: ROWS rows).  The layout is
+// the one a TMA box load with hardware swizzling produces, so that K/V tiles can arrive either way: rows of at most
+// 128 bytes (head_dim 128 = two column halves of 64, stored one after the other), 16-byte chunks XOR-ed with the
+// row index (128-byte swizzle; 64-byte swizzle for head_dim 32).  The XOR also keeps the eight rows of an ldmatrix
+// phase on distinct banks.  Tile bases are 1024-byte aligned.
+template <int HD, int ROWS = 64>
 __device__ __forceinline__ uint32_t swz(int row, int chunk) {
-    constexpr int RB = HD * 2;
-    if (RB >= 128) return (uint32_t)(row * RB + ((chunk ^ (row & 7)) << 4));
-    return (uint32_t)(row * RB + ((chunk ^ ((row >> 1) & 3)) << 4));
+    if (HD == 128) return (uint32_t)((chunk >> 3) * (ROWS * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+    if (HD == 64) return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
+    return (uint32_t)(row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4));
 }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
@@ -101,19 +108,21 @@ __device__ __forceinline__ void cp_async_wait_dyn(int n) {      // wait until at
 
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32)
-attn_mma_kernel(const AttnArgs a) {
+attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
     constexpr int GP = NW * 16;                  // padded query rows
     constexpr int CH = HD / 8;                   // 16-byte chunks per row
     constexpr int THREADS = NW * 32;
     constexpr int TILE_BYTES = TKEYS * HD * 2;
     const int STAGES = a.stages;                 // ring depth of this launch, 2 .. Ring<HD, NW>::MAX_STAGES
-    extern __shared__ __align__(128) uint8_t sm[];
+    extern __shared__ uint8_t sm_raw[];
+    uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // swizzled tiles sit on 1024-byte boundaries
     uint8_t* Qh = sm;
     uint8_t* Ql = Qh + GP * HD * 2;
     uint8_t* Kt = Ql + GP * HD * 2;              // [STAGES][TKEYS][HD]
     uint8_t* Vt = Kt + STAGES * TILE_BYTES;      // [STAGES][TKEYS][HD]
     constexpr int MAX_STAGED_PAGES = 1024;
     __shared__ int s_pages[MAX_STAGED_PAGES];
+    __shared__ uint64_t s_full[8];               // one per ring stage: bytes of its K and V tile have landed (TMA path)
 
     const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -163,16 +172,45 @@ attn_mma_kernel(const AttnArgs a) {
     const int pg_lo = k_begin / a.page_size;
     const int n_pg = n_tiles > 0 ? (k_end - 1) / a.page_size - pg_lo + 1 : 0;
     const bool pages_staged = n_pg <= MAX_STAGED_PAGES;
+    const bool use_tma = a.use_tma && pages_staged;
+    if (tid == 0 && use_tma) {
+        for (int i = 0; i < STAGES; ++i) mbar_init(smem_u32(&s_full[i]), 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+    }
     if (pages_staged) {
         for (int i = tid; i < n_pg; i += THREADS) {
             const int pslot = pg_lo + i;
             int page = -1;
             if (pslot < a.max_pages) page = a.block_table[(size_t)b * a.max_pages + pslot];
-            s_pages[i] = (page >= 0 && page < a.n_pages) ? page : -1;      // ids outside the pool read as zeros, never as memory
+            s_pages[i] = (page >= 0 && page < a.n_pages) ? page : -1;      // ids outside the pool are never used as addresses
         }
-        __syncthreads();
     }
-    // One row of the tile per TPR threads: a page lookup, then the thread's share of the row's 16-byte chunks.
+    __syncthreads();
+    // TMA path (thread 0): a tile is four 16-token pages; each page of this KV head is one box (two for head_dim
+    // 128) of the [pages * kv_heads * 16][head_dim] view of the pool.  Rows past the key range re-read the range's
+    // last page and a page id outside the pool reads page 0: both are masked later, and nothing unmapped is touched.
+    auto load_tile_tma = [&](int tile, int stage) {
+        const uint32_t bar = smem_u32(&s_full[stage]);
+        const uint32_t kdst = smem_u32(Kt + stage * TILE_BYTES), vdst = smem_u32(Vt + stage * TILE_BYTES);
+        mbar_expect_tx(bar, 2u * TILE_BYTES);
+#pragma unroll
+        for (int pg = 0; pg < TKEYS / 16; ++pg) {
+            int key = k_begin + tile * TKEYS + pg * 16;
+            key = key < k_end ? key : k_end - 1;
+            int page = s_pages[key / 16 - pg_lo];
+            page = page < 0 ? 0 : page;
+            const int y = (page * a.n_kv + kh) * 16;
+            constexpr int BOXB = (HD >= 64 ? 128 : 64) * 16;       // bytes of one box: 16 rows of at most 128 bytes
+#pragma unroll
+            for (int h = 0; h < (HD == 128 ? 2 : 1); ++h) {
+                tma_load_2d(kdst + h * (TKEYS * 128) + pg * BOXB, &tmK, h * 64, y, bar);
+                tma_load_2d(vdst + h * (TKEYS * 128) + pg * BOXB, &tmV, h * 64, y, bar);
+            }
+        }
+    };
+    // cp.async path: one row of the tile per TPR threads: a page lookup, then the thread's share of the row's chunks.
     constexpr int TPR = THREADS / TKEYS, CPT = CH / TPR;
     auto load_tile = [&](int tile, int stage) {
         const int row = tid / TPR, c0 = (tid % TPR) * CPT;
@@ -196,14 +234,20 @@ attn_mma_kernel(const AttnArgs a) {
 #pragma unroll
         for (int j = 0; j < CPT; ++j) {
             const uint32_t so = swz<HD>(row, c0 + j);
-            cp_async16(kdst + so, a.kp + off + (c0 + j) * 8, bytes);
+            cp_async16(kdst + so, a.kp + off + (c0 + j) * 8, bytes);     // zero-fills when bytes = 0
             cp_async16(vdst + so, a.vp + off + (c0 + j) * 8, bytes);
         }
     };
-    auto load_super = [&](int sup) {                             // the ng tiles of iteration `sup`, one commit group
-        for (int j = 0; j < ng; ++j)
-            if (sup * ng + j < n_tiles) load_tile(sup * ng + j, (sup % super_stages) * ng + j);
-        cp_async_commit();
+    auto load_super = [&](int sup) {                             // the ng tiles of iteration `sup`
+        if (use_tma) {
+            if (tid == 0)
+                for (int j = 0; j < ng; ++j)
+                    if (sup * ng + j < n_tiles) load_tile_tma(sup * ng + j, (sup % super_stages) * ng + j);
+        } else {
+            for (int j = 0; j < ng; ++j)
+                if (sup * ng + j < n_tiles) load_tile(sup * ng + j, (sup % super_stages) * ng + j);
+            cp_async_commit();                                   // one group per iteration, empty past the end
+        }
     };
     // prologue of the ring: tiles that lie wholly inside the committed prefix start before the wait,
     // the tiles holding this step's new rows (written by the preceding grid) after it
@@ -240,7 +284,7 @@ attn_mma_kernel(const AttnArgs a) {
         uint2 h, l;
         pack_hilo(v.x, v.y, h.x, l.x);
         pack_hilo(v.z, v.w, h.y, l.y);
-        const uint32_t so = swz<HD>(rho, d4 >> 3) + (uint32_t)((d4 & 7) * 2);
+        const uint32_t so = swz<HD, GP>(rho, d4 >> 3) + (uint32_t)((d4 & 7) * 2);
         *reinterpret_cast<uint2*>(Qh + so) = h;
         *reinterpret_cast<uint2*>(Ql + so) = l;
     }
@@ -260,8 +304,15 @@ attn_mma_kernel(const AttnArgs a) {
 
     for (int sup = 0; sup < n_super; ++sup) {
         if (sup + super_stages - 1 < n_super) load_super(sup + super_stages - 1);
-        else cp_async_commit();
-        cp_async_wait_dyn(super_stages - 1);                      // iteration `sup` has landed
+        else if (!use_tma) cp_async_commit();
+        if (use_tma) {                                             // iteration `sup` has landed (bounded wait)
+            for (int j = 0; j < ng; ++j)
+                if (sup * ng + j < n_tiles &&
+                    !mbar_wait(smem_u32(&s_full[(sup % super_stages) * ng + j]), (uint32_t)(sup / super_stages) & 1u))
+                    set_status(a.status, TASC_ETIMEOUT);
+        } else {
+            cp_async_wait_dyn(super_stages - 1);
+        }
         __syncthreads();
 #ifdef TASC_TIMELINE
         if (sup == 0) log_at_exit.td = global_ns();
@@ -280,7 +331,7 @@ attn_mma_kernel(const AttnArgs a) {
 #pragma unroll
             for (int ks = 0; ks < HD / 16; ++ks) {
                 uint32_t qh[4], ql[4];
-                const uint32_t qo = swz<HD>(slab * 16 + (mi & 1) * 8 + li, ks * 2 + (mi >> 1));
+                const uint32_t qo = swz<HD, GP>(slab * 16 + (mi & 1) * 8 + li, ks * 2 + (mi >> 1));
                 ldsm_x4(qh_base + qo, qh);
                 ldsm_x4(ql_base + qo, ql);
                 // eight independent accumulators between two MMAs on the same one (hi pass, then lo pass)
@@ -490,7 +541,7 @@ attn_mma_kernel(const AttnArgs a) {
 }
 
 inline size_t attn_smem_bytes(int hd, int gp, int stages) {
-    return (size_t)2 * gp * hd * 2 + (size_t)2 * stages * TKEYS * hd * 2;
+    return 1024 + (size_t)2 * gp * hd * 2 + (size_t)2 * stages * TKEYS * hd * 2;      // 1024: alignment slack
 }
 
 template <int HD, int NW>
@@ -543,7 +594,7 @@ int fit_any(int hd, int nw, int splits, int stages) {
 }
 
 template <int HD, int NW>
-tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
+tasc_status launch_inst(const AttnArgs& a, const CUtensorMap& tmK, const CUtensorMap& tmV, int B, cudaStream_t stream) {
     constexpr int GP = NW * 16;
     if (a.stages < 2 || a.stages > Ring<HD, NW>::MAX_STAGES) return TASC_EINVAL;
     const size_t smem = attn_smem_bytes(HD, GP, a.stages);
@@ -568,7 +619,7 @@ tasc_status launch_inst(const AttnArgs& a, int B, cudaStream_t stream) {
     cfg.attrs = at;
     cfg.numAttrs = n_at;
     ProfScope ps(K_ATT_SPLIT, stream);
-    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_mma_kernel<HD, NW>, a));
+    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_mma_kernel<HD, NW>, tmK, tmV, a));
     return TASC_OK;
 }
 
@@ -608,7 +659,7 @@ AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx) {
 tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
                                  const int32_t* block_table, int max_pages, int page_size, long long n_pages,
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
-                                 const AttnPlan& plan, cudaStream_t stream) {
+                                 const AttnPlan& plan, int* status, cudaStream_t stream) {
     const int n_splits = plan.splits;
     const int G = (n_q / n_kv) * R;
     if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 8) return TASC_EINVAL;
@@ -620,14 +671,26 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
     a.out = out; a.TB = TB;
     a.R = R; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits; a.stages = plan.stages;
     a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
-    if (GP == 64) {
-        if (hd == 32) return launch_inst<32, 4>(a, B, stream);
-        if (hd == 64) return launch_inst<64, 4>(a, B, stream);
-        return launch_inst<128, 4>(a, B, stream);
+    a.status = status;
+    // 16-token pages arrive as TMA boxes; any other page size takes the cp.async path of the same kernel
+    a.use_tma = page_size == 16 ? 1 : 0;
+    CUtensorMap tmK, tmV;
+    memset(&tmK, 0, sizeof(tmK));
+    memset(&tmV, 0, sizeof(tmV));
+    if (a.use_tma) {
+        const uint64_t rows = (uint64_t)n_pages * n_kv * 16;
+        tasc_status st;
+        if ((st = encode_tmap_kv(&tmK, k_pages, rows, hd)) != TASC_OK) return st;
+        if ((st = encode_tmap_kv(&tmV, v_pages, rows, hd)) != TASC_OK) return st;
     }
-    if (hd == 32) return launch_inst<32, 8>(a, B, stream);
-    if (hd == 64) return launch_inst<64, 8>(a, B, stream);
-    return launch_inst<128, 8>(a, B, stream);
+    if (GP == 64) {
+        if (hd == 32) return launch_inst<32, 4>(a, tmK, tmV, B, stream);
+        if (hd == 64) return launch_inst<64, 4>(a, tmK, tmV, B, stream);
+        return launch_inst<128, 4>(a, tmK, tmV, B, stream);
+    }
+    if (hd == 32) return launch_inst<32, 8>(a, tmK, tmV, B, stream);
+    if (hd == 64) return launch_inst<64, 8>(a, tmK, tmV, B, stream);
+    return launch_inst<128, 8>(a, tmK, tmV, B, stream);
 }
 
 }  // namespace tasc

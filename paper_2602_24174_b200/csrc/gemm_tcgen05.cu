@@ -202,6 +202,20 @@ tasc_status encode_tmap_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, u
     return r == CUDA_SUCCESS ? TASC_OK : TASC_ECUDA;
 }
 
+tasc_status encode_tmap_kv(CUtensorMap* map, const void* ptr, uint64_t rows, int hd) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return TASC_ECUDA;
+    if ((reinterpret_cast<uintptr_t>(ptr) & 15u) || (hd != 32 && hd != 64 && hd != 128) || rows == 0) return TASC_EINVAL;
+    cuuint64_t dims[2] = {(cuuint64_t)hd, rows};
+    cuuint64_t strides[1] = {(cuuint64_t)hd * 2};
+    cuuint32_t box[2] = {(cuuint32_t)(hd < 64 ? hd : 64), 16};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, hd < 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TASC_OK : TASC_ECUDA;
+}
+
 int gemm_token_tile(int M, bool pair) {
     const int cap = pair ? 128 : 256;                 // tokens per tile (UMMA N <= 256)
     const int m_tiles = (M + cap - 1) / cap;

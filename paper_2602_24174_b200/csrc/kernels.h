@@ -36,6 +36,9 @@ inline size_t gemm_partial_bytes(const GemmPlan& p, int M, int N) { return (size
 
 // rows x cols bf16 row-major matrix, box = {64 cols, box_rows}, 128-byte swizzle.
 tasc_status encode_tmap_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// One layer's K (or V) pages seen as a rows x head_dim bf16 matrix (rows = pages * kv_heads * 16): box = one page of
+// one KV head, {min(head_dim, 64) columns, 16 rows}, 128-byte swizzle (64-byte for head_dim 32).
+tasc_status encode_tmap_kv(CUtensorMap* map, const void* ptr, uint64_t rows, int hd);
 
 tasc_status launch_gemm_bf16(const CUtensorMap* tmW, const CUtensorMap* tmX, float* partials, int M, int N, int K,
                              const GemmPlan& plan, int* status, cudaStream_t stream);
@@ -165,7 +168,7 @@ struct AttnPlan {
 tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
                                  const int32_t* block_table, int max_pages, int page_size, long long n_pages,
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
-                                 const AttnPlan& plan, cudaStream_t stream);
+                                 const AttnPlan& plan, int* status, cudaStream_t stream);
 AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx);
 
 }  // namespace tasc
