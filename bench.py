@@ -383,8 +383,12 @@ def main():
             gt[:, :P] = torch.from_numpy(prompts).to(dev)
             gl = torch.full((B,), P, dtype=torch.int32, device=dev)
             gpool, gbt, gkv = model.new_kv(B, gstride + b.MAX_ROWS, dev)
-            _, st = b.tasc_generate(model, drafter, gkv, b.make_seqs(gt, gl), B, max_new, k, ws, lambda_num=cfg.lambda_num,
-                                    lambda_den=cfg.lambda_den, mode=mode, forced_accept=forced_accept, continuation=cont)
+            gen_stream = torch.cuda.Stream(device=dev)              # not the default stream: the loop replays a CUDA graph
+            gen_stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(gen_stream):
+                _, st = b.tasc_generate(model, drafter, gkv, b.make_seqs(gt, gl), B, max_new, k, ws, lambda_num=cfg.lambda_num,
+                                        lambda_den=cfg.lambda_den, mode=mode, forced_accept=forced_accept, continuation=cont)
+            torch.cuda.current_stream().wait_stream(gen_stream)
             hist = list(st.accepted_hist)[:k + 1]
             seq_steps = max(sum(hist), 1)
             return {"tokens_per_s": B * max_new / (st.decode_ms * 1e-3), "decode_ms": st.decode_ms, "prefill_ms": st.prefill_ms,

@@ -223,6 +223,8 @@ typedef struct {
  * on return tokens/len hold prompt + generated tokens (a sequence may overshoot max_new by up to k).
  *   out    device, int32[B][max_new] (written): the first max_new generated tokens
  *   stats  host (written), may be NULL
+ * On a stream other than the legacy default stream the step is captured once into a CUDA graph (after a first
+ * plainly enqueued step) and replayed, which allocates the graph's resources for the duration of the call.
  * Synchronises the stream.  Errors: EINVAL, ECUDA, and device-side statuses (ENOKV, ETIMEOUT).
  */
 tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* d, const tasc_kv* kv, const tasc_seqs* seqs,

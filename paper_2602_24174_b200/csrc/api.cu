@@ -409,16 +409,37 @@ extern "C" tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* dr
     int64_t steps = 0;
     int min_gen = 0;
     const bool forced = p->mode != TASC_MODE_GREEDY;
+    auto enqueue_step = [&]() -> tasc_status {
+        tasc_status e = tasc_draft(dr, seqs.tokens, seqs.stride, seqs.len, B, k, p->lambda_num, p->lambda_den, w.drafts, s);
+        if (e != TASC_OK) return e;
+        if (forced)
+            launch_forced_targets(p->mode, w.drafts, p->continuation, p->continuation_stride, seqs.len, w.prompt_len,
+                                  p->forced_accept, m->desc.vocab, B, k, w.targets, s);
+        return verify_enqueue(m, kv, &seqs, w, w.drafts, B, k, forced ? w.targets : nullptr, w.n_accepted, w.next_token,
+                              nullptr, nullptr, s);
+    };
+    // Every step enqueues the same ~5 launches per layer on the same buffers, so after a first plain step the step
+    // is captured once into a CUDA graph and replayed: the host then costs one launch per step instead of ~150.
+    // (Not possible on the legacy default stream, and not while launch timing is on: then every step is enqueued.)
+    cudaGraphExec_t step_graph = nullptr;
+    auto capture_step = [&]() {
+        if (s == nullptr || s == cudaStreamLegacy || profiling_enabled()) return;
+        if (cudaStreamBeginCapture(s, cudaStreamCaptureModeRelaxed) != cudaSuccess) { (void)cudaGetLastError(); return; }
+        const tasc_status e = enqueue_step();
+        cudaGraph_t g = nullptr;
+        if (cudaStreamEndCapture(s, &g) != cudaSuccess || e != TASC_OK || !g) { (void)cudaGetLastError(); if (g) cudaGraphDestroy(g); return; }
+        if (cudaGraphInstantiate(&step_graph, g, 0) != cudaSuccess) { (void)cudaGetLastError(); step_graph = nullptr; }
+        cudaGraphDestroy(g);
+    };
     while (st == TASC_OK && min_gen < max_new) {
         const int todo = (max_new - min_gen + k) / (k + 1);      // the slowest sequence needs at least this many steps
         for (int i = 0; i < todo && st == TASC_OK; ++i) {
-            st = tasc_draft(dr, seqs.tokens, seqs.stride, seqs.len, B, k, p->lambda_num, p->lambda_den, w.drafts, s);
-            if (st != TASC_OK) break;
-            if (forced)
-                launch_forced_targets(p->mode, w.drafts, p->continuation, p->continuation_stride, seqs.len, w.prompt_len,
-                                      p->forced_accept, m->desc.vocab, B, k, w.targets, s);
-            st = verify_enqueue(m, kv, &seqs, w, w.drafts, B, k, forced ? w.targets : nullptr, w.n_accepted, w.next_token,
-                                nullptr, nullptr, s);
+            if (steps == 1 && !step_graph) capture_step();       // step 0 ran plainly (first-use set-up happens outside a capture)
+            if (step_graph && steps >= 1) {
+                if (cudaGraphLaunch(step_graph, s) != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; }
+            } else {
+                st = enqueue_step();
+            }
             ++steps;
         }
         if (st != TASC_OK) break;
@@ -429,6 +450,7 @@ extern "C" tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* dr
         if (cudaMemcpy(&dev_status, w.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { (void)cudaGetLastError(); st = TASC_ECUDA; break; }
         if (dev_status != 0) { st = dev_status; break; }
     }
+    if (step_graph) cudaGraphExecDestroy(step_graph);
     cudaEventRecord(ev[2], s);
     if (st == TASC_OK) {
         launch_gather_output(seqs.tokens, seqs.stride, w.prompt_len, B, max_new, out, s);

@@ -10,6 +10,7 @@ enum Kind { K_DRAFT, K_ROWS, K_EMBED, K_GEMM, K_GEMM_LM, K_QKV_ROPE, K_ATT_SPLIT
             K_ACCEPT, K_OTHER, K_COUNT };
 void prof_begin(int kind, cudaStream_t s);     // counts the launch; records an event when timing is enabled
 void prof_end(int kind, cudaStream_t s);
+bool profiling_enabled();                      // per-launch event timing is on (tasc_profile_enable)
 struct ProfScope {
     int kind; cudaStream_t s;
     ProfScope(int k, cudaStream_t st) : kind(k), s(st) { prof_begin(kind, s); }

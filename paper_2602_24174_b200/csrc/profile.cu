@@ -46,6 +46,8 @@ void note_cuda_error(cudaError_t e, const char* expr, const char* file, int line
     snprintf(g_last_error, sizeof(g_last_error), "%s (%s) at %s:%d in `%s`", cudaGetErrorName(e), cudaGetErrorString(e), base, line, expr);
 }
 
+bool profiling_enabled() { return g_enabled.load(std::memory_order_relaxed) != 0; }
+
 void prof_begin(int kind, cudaStream_t s) {
     g_launches[kind].fetch_add(1, std::memory_order_relaxed);
     t_open[kind] = nullptr;

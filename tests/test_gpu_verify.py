@@ -51,7 +51,8 @@ def test_config0_teacher_forced_accept_lengths():
 
 
 @pytest.mark.gpu
-def test_config0_generate_matches_oracle_and_plain_greedy():
+@pytest.mark.parametrize("side_stream", [False, True])      # a non-default stream makes tasc_generate replay a CUDA graph
+def test_config0_generate_matches_oracle_and_plain_greedy(side_stream):
     b = need_gpu()
     cfg = configs.get(0)
     s = make_setup(cfg)
@@ -64,7 +65,11 @@ def test_config0_generate_matches_oracle_and_plain_greedy():
     length = torch.full((B,), P, dtype=torch.int32, device="cuda")
     pool, bt, kv = s.model.new_kv(B, stride + b.MAX_ROWS)
     ws = s.model.new_workspace(B, cfg.k)
-    out, st = b.tasc_generate(s.model, s.drafter, kv, b.make_seqs(tokens, length), B, cfg.max_new, cfg.k, ws)
+    stream = torch.cuda.Stream() if side_stream else torch.cuda.current_stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        out, st = b.tasc_generate(s.model, s.drafter, kv, b.make_seqs(tokens, length), B, cfg.max_new, cfg.k, ws)
+    torch.cuda.current_stream().wait_stream(stream)
     out = out.cpu().numpy()
     assert st.steps >= cfg.max_new // (cfg.k + 1) and st.committed >= B * cfg.max_new
     assert sum(st.accepted_hist) > 0 and st.decode_ms > 0
@@ -204,3 +209,30 @@ def test_config2_batch32_k3_and_k8_one_step():
     prompts = corpus.make_prompts(cfg, 32, prompt_len=80)
     for k in (3, 8):
         check(lockstep(s, prompts, k + 1, k, **BF16_TOL))
+
+
+@pytest.mark.gpu
+def test_config1_generate_graph_replay_equals_plain_enqueue(setup1):
+    """tasc_generate on a side stream (captured step replayed from a CUDA graph) must produce exactly the tokens and
+    statistics of the same call on the default stream (every step enqueued)."""
+    b = need_gpu()
+    cfg = configs.get(1)
+    B, max_new, k = 3, 40, cfg.k
+    prompts = corpus.make_prompts(cfg, B)
+    P = prompts.shape[1]
+    results = []
+    for side in (False, True):
+        stride = P + max_new + k + 2
+        tokens = torch.zeros((B, stride), dtype=torch.int32, device="cuda")
+        tokens[:, :P] = torch.from_numpy(prompts).cuda()
+        length = torch.full((B,), P, dtype=torch.int32, device="cuda")
+        pool, bt, kv = setup1.model.new_kv(B, stride + b.MAX_ROWS)
+        ws = setup1.model.new_workspace(B, k)
+        stream = torch.cuda.Stream() if side else torch.cuda.current_stream()
+        stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(stream):
+            out, st = b.tasc_generate(setup1.model, setup1.drafter, kv, b.make_seqs(tokens, length), B, max_new, k, ws)
+        torch.cuda.current_stream().wait_stream(stream)
+        results.append((out.cpu().numpy(), st.steps, list(st.accepted_hist)))
+    assert np.array_equal(results[0][0], results[1][0])
+    assert results[0][1:] == results[1][1:]
