@@ -235,6 +235,17 @@ tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* d, const tasc
 tasc_status tasc_poll_status(void* workspace, tasc_stream stream);
 
 /*
+ * Failure-path self-test.  Every device-side wait of the library (TMA arrival, MMA completion, ring slots) is
+ * bounded: when the budget runs out the kernel records TASC_ETIMEOUT in the status word, gives up the wait and
+ * returns normally, so the context stays usable.  This call launches a one-thread kernel that waits, through the
+ * same routine, on a barrier that nothing will ever signal, for budget_cycles SM clock cycles (1 .. 2e9); a following
+ * tasc_poll_status(workspace) must then report TASC_ETIMEOUT.  Nothing faults or hangs.
+ *   workspace  device, at least 4 bytes: the status word
+ * Asynchronous.  Errors: EINVAL.
+ */
+tasc_status tasc_selftest_bounded_wait(void* workspace, int64_t budget_cycles, tasc_stream stream);
+
+/*
  * Y[M][N] (float32) = X[M][K] * W[N][K]^T for bf16 X and W on the tensor cores, the building block of
  * every projection of the verify forward (exported for unit tests and profiling).
  *   x, w       device, bf16, row-major, 16-byte aligned; K a multiple of 8

@@ -88,6 +88,8 @@ lib.tasc_verify_step.argtypes = [_P, C.POINTER(Kv), C.POINTER(Seqs), _P, C.c_int
 lib.tasc_generate.argtypes = [_P, _P, C.POINTER(Kv), C.POINTER(Seqs), C.c_int32, C.c_int32, C.POINTER(DraftParams), _P,
                               C.POINTER(Stats), _P, C.c_size_t, _P]
 lib.tasc_poll_status.argtypes = [_P, _P]
+lib.tasc_selftest_bounded_wait.argtypes = [_P, C.c_int64, _P]
+lib.tasc_selftest_bounded_wait.restype = C.c_int32
 lib.tasc_gemm_bf16.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 lib.tasc_gemm_bf16x2.argtypes = [_P, _P, _P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_size_t, _P]
 lib.tasc_gemm_bf16x2.restype = C.c_int32
@@ -279,6 +281,11 @@ def tasc_generate(model: Model, drafter: Drafter, kv: Kv, seqs: Seqs, B: int, ma
 
 def tasc_poll_status(workspace: torch.Tensor):
     _check(lib.tasc_poll_status(_ptr(workspace), _stream()), "tasc_poll_status")
+
+
+def tasc_selftest_bounded_wait(workspace: torch.Tensor, budget_cycles: int = 200_000):
+    """Launches the kernel that waits on a never-signalled barrier; tasc_poll_status(workspace) then raises ETIMEOUT."""
+    _check(lib.tasc_selftest_bounded_wait(_ptr(workspace), budget_cycles, _stream()), "tasc_selftest_bounded_wait")
 
 
 def tasc_gemm_bf16(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:

@@ -485,6 +485,13 @@ extern "C" tasc_status tasc_poll_status(void* workspace, tasc_stream stream) {
     return v;
 }
 
+extern "C" tasc_status tasc_selftest_bounded_wait(void* workspace, int64_t budget_cycles, tasc_stream stream) {
+    if (!workspace || budget_cycles < 1 || budget_cycles > 2000000000ll) return TASC_EINVAL;
+    launch_wait_selftest(budget_cycles, static_cast<int*>(workspace), static_cast<cudaStream_t>(stream));
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
 extern "C" size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K) {
     if (M < 1 || N < 1 || K < 1) return 0;
     const GemmPlan p = plan_gemm(M, N, K, (size_t)1 << 40, false);

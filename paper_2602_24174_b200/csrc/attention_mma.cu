@@ -91,7 +91,15 @@ __device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32
 // Largest ring depth of the K/V tile pipeline (the host picks 2..max per launch).  A CTA streams its key range
 // alone, so the bytes it keeps in flight (ring depth x 8-32 KB per tile) over the memory latency are its
 // bandwidth; a shallower ring lets two CTAs share an SM when many (sequence, KV head) pairs are in flight.
-template <int HD, int NW> struct Ring { static constexpr int MAX_STAGES = HD >= 128 ? (NW > 4 ? 4 : 5) : 8; };
+template <int HD, int NS> struct Ring { static constexpr int MAX_STAGES = HD >= 128 ? (NS > 4 ? 4 : 5) : 8; };
+
+// Warp groups of an eight-warp CTA whose query tile has n_slabs slabs (each group needs two ring stages).
+__host__ __device__ inline int warp_groups(int n_slabs, int stages) {
+    int ng = 8 / n_slabs;
+    ng = ng >= 4 ? 4 : (ng >= 2 ? 2 : 1);
+    while (ng > 1 && stages / ng < 2) ng >>= 1;
+    return ng;
+}
 
 __device__ __forceinline__ void cp_async_wait_dyn(int n) {      // wait until at most n groups are pending
     switch (n) {
@@ -106,14 +114,16 @@ __device__ __forceinline__ void cp_async_wait_dyn(int n) {      // wait until at
     }
 }
 
-template <int HD, int NW>
-__global__ void __launch_bounds__(NW * 32)
+// NS = number of 16-row slabs the padded query tile has (4 or 8); the CTA always has eight warps.
+template <int HD, int NS>
+__global__ void __launch_bounds__(256)
 attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const AttnArgs a) {
-    constexpr int GP = NW * 16;                  // padded query rows
+    constexpr int NW = 8;                        // warps
+    constexpr int GP = NS * 16;                  // padded query rows
     constexpr int CH = HD / 8;                   // 16-byte chunks per row
     constexpr int THREADS = NW * 32;
     constexpr int TILE_BYTES = TKEYS * HD * 2;
-    const int STAGES = a.stages;                 // ring depth of this launch, 2 .. Ring<HD, NW>::MAX_STAGES
+    const int STAGES = a.stages;                 // ring depth of this launch, 2 .. Ring<HD, NS>::MAX_STAGES
     extern __shared__ uint8_t sm_raw[];
     uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // swizzled tiles sit on 1024-byte boundaries
     uint8_t* Qh = sm;
@@ -160,9 +170,9 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int k_end = min(total, k_begin + chunk);
     const int n_tiles = k_begin < k_end ? (k_end - k_begin + TKEYS - 1) / TKEYS : 0;
     const int n_slabs = (G + 15) / 16;
-    // With few query rows the spare warps take every other key tile: warp group `grp` (n_slabs warps,
-    // one 16-row slab each) handles tiles grp, grp + ng, ...; the groups' results are merged in shared memory.
-    const int ng = (STAGES >= 4 && NW / n_slabs >= 2) ? 2 : 1;
+    // A warp owns one 16-row slab of one key tile.  With fewer slabs than warps the warps form ng = 2 or 4 groups
+    // of n_slabs warps; group `grp` handles tiles grp, grp + ng, ...; the groups' results are merged in shared memory.
+    const int ng = warp_groups(n_slabs, STAGES);
     const int slab = warp % n_slabs, grp = warp / n_slabs;
     const bool computes = grp < ng;
     const int n_super = (n_tiles + ng - 1) / ng;                 // iterations of ng tiles
@@ -420,27 +430,32 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], 1);
         l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], 2);
     }
-    if (ng == 2) {
-        // second warp group -> shared memory (the K/V ring is idle) -> first group folds it into its own state
-        float* xg = reinterpret_cast<float*>(Kt) + (size_t)(slab * 32 + lane) * (HD / 2 + 4);
-        if (computes && grp == 1) {
+    if (ng > 1) {
+        // groups 1 .. ng-1 -> shared memory (the K/V ring is idle) -> group 0 folds them into its state, in group order
+        constexpr int XG = HD / 2 + 4;                          // floats per lane: O fragment, two maxima, two sums
+        float* xg0 = reinterpret_cast<float*>(Kt);
+        if (computes && grp > 0) {
+            float* xg = xg0 + ((size_t)((grp - 1) * n_slabs + slab) * 32 + lane) * XG;
 #pragma unroll
             for (int i = 0; i < HD / 8; ++i) { xg[4 * i] = o[i][0]; xg[4 * i + 1] = o[i][1]; xg[4 * i + 2] = o[i][2]; xg[4 * i + 3] = o[i][3]; }
             xg[HD / 2] = m_run[0]; xg[HD / 2 + 1] = m_run[1]; xg[HD / 2 + 2] = l_run[0]; xg[HD / 2 + 3] = l_run[1];
         }
         __syncthreads();
         if (grp == 0) {
-            const float om0 = xg[HD / 2], om1 = xg[HD / 2 + 1], ol0 = xg[HD / 2 + 2], ol1 = xg[HD / 2 + 3];
-            const float mn0 = fmaxf(m_run[0], om0), mn1 = fmaxf(m_run[1], om1);
-            const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
-            const float sa0 = exp2f(m_run[0] - mu0), sb0 = exp2f(om0 - mu0), sa1 = exp2f(m_run[1] - mu1), sb1 = exp2f(om1 - mu1);
+            for (int og = 1; og < ng; ++og) {
+                const float* xg = xg0 + ((size_t)((og - 1) * n_slabs + slab) * 32 + lane) * XG;
+                const float om0 = xg[HD / 2], om1 = xg[HD / 2 + 1], ol0 = xg[HD / 2 + 2], ol1 = xg[HD / 2 + 3];
+                const float mn0 = fmaxf(m_run[0], om0), mn1 = fmaxf(m_run[1], om1);
+                const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+                const float sa0 = exp2f(m_run[0] - mu0), sb0 = exp2f(om0 - mu0), sa1 = exp2f(m_run[1] - mu1), sb1 = exp2f(om1 - mu1);
 #pragma unroll
-            for (int i = 0; i < HD / 8; ++i) {
-                o[i][0] = o[i][0] * sa0 + xg[4 * i] * sb0;     o[i][1] = o[i][1] * sa0 + xg[4 * i + 1] * sb0;
-                o[i][2] = o[i][2] * sa1 + xg[4 * i + 2] * sb1; o[i][3] = o[i][3] * sa1 + xg[4 * i + 3] * sb1;
+                for (int i = 0; i < HD / 8; ++i) {
+                    o[i][0] = o[i][0] * sa0 + xg[4 * i] * sb0;     o[i][1] = o[i][1] * sa0 + xg[4 * i + 1] * sb0;
+                    o[i][2] = o[i][2] * sa1 + xg[4 * i + 2] * sb1; o[i][3] = o[i][3] * sa1 + xg[4 * i + 3] * sb1;
+                }
+                l_run[0] = l_run[0] * sa0 + ol0 * sb0; l_run[1] = l_run[1] * sa1 + ol1 * sb1;
+                m_run[0] = mn0; m_run[1] = mn1;
             }
-            l_run[0] = l_run[0] * sa0 + ol0 * sb0; l_run[1] = l_run[1] * sa1 + ol1 * sb1;
-            m_run[0] = mn0; m_run[1] = mn1;
         }
     }
     const bool writer = computes && grp == 0;                  // holds the CTA's result for its slab
@@ -544,27 +559,27 @@ inline size_t attn_smem_bytes(int hd, int gp, int stages) {
     return 1024 + (size_t)2 * gp * hd * 2 + (size_t)2 * stages * TKEYS * hd * 2;      // 1024: alignment slack
 }
 
-template <int HD, int NW>
+template <int HD, int NS>
 tasc_status prepare_inst() {
     static bool done[64] = {false};
     int dev = 0;
     TASC_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return TASC_EINVAL;
     if (!done[dev]) {
-        TASC_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<HD, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        TASC_CUDA_TRY(cudaFuncSetAttribute(attn_mma_kernel<HD, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
         done[dev] = true;
     }
     return TASC_OK;
 }
 
 // Clusters of `splits` CTAs (ring depth `stages`) the device holds at once; 0 if the query fails.
-template <int HD, int NW>
+template <int HD, int NS>
 int fit_inst(int splits, int stages) {
-    if (prepare_inst<HD, NW>() != TASC_OK) return 0;
+    if (prepare_inst<HD, NS>() != TASC_OK) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)splits, 1, 1);
-    cfg.blockDim = dim3(NW * 32, 1, 1);
-    cfg.dynamicSmemBytes = attn_smem_bytes(HD, NW * 16, stages);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = attn_smem_bytes(HD, NS * 16, stages);
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)splits;
@@ -573,7 +588,7 @@ int fit_inst(int splits, int stages) {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, attn_mma_kernel<HD, NW>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    if (cudaOccupancyMaxActiveClusters(&n, attn_mma_kernel<HD, NS>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
     return n;
 }
 
@@ -593,16 +608,16 @@ int fit_any(int hd, int nw, int splits, int stages) {
     return n;
 }
 
-template <int HD, int NW>
+template <int HD, int NS>
 tasc_status launch_inst(const AttnArgs& a, const CUtensorMap& tmK, const CUtensorMap& tmV, int B, cudaStream_t stream) {
-    constexpr int GP = NW * 16;
-    if (a.stages < 2 || a.stages > Ring<HD, NW>::MAX_STAGES) return TASC_EINVAL;
+    constexpr int GP = NS * 16;
+    if (a.stages < 2 || a.stages > Ring<HD, NS>::MAX_STAGES) return TASC_EINVAL;
     const size_t smem = attn_smem_bytes(HD, GP, a.stages);
-    tasc_status pst = prepare_inst<HD, NW>();
+    tasc_status pst = prepare_inst<HD, NS>();
     if (pst != TASC_OK) return pst;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)a.splits, (unsigned)a.n_kv, (unsigned)B);
-    cfg.blockDim = dim3(NW * 32, 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute at[2];
@@ -619,7 +634,7 @@ tasc_status launch_inst(const AttnArgs& a, const CUtensorMap& tmK, const CUtenso
     cfg.attrs = at;
     cfg.numAttrs = n_at;
     ProfScope ps(K_ATT_SPLIT, stream);
-    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_mma_kernel<HD, NW>, tmK, tmV, a));
+    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_mma_kernel<HD, NS>, tmK, tmV, a));
     return TASC_OK;
 }
 
@@ -628,28 +643,28 @@ tasc_status launch_inst(const AttnArgs& a, const CUtensorMap& tmK, const CUtenso
 int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
 
 // Key-range splits per (sequence, KV head) (1..8, the CTAs of a cluster) and ring depth, from a small cost model
-// in microseconds: a CTA needs about 1.5 us to start plus one tile time per iteration (its warp groups take `ng`
+// in microseconds: a CTA needs about 2.5 us to start (Q staging, first tiles) plus one tile time per iteration (its warp groups take `ng`
 // tiles per iteration; a shallow ring adds memory stalls), the clusters run in as many waves as the device's
 // cluster occupancy dictates (one straggling cluster costs a whole wave), and splitting adds the cluster
 // exchange and merge (about 4.5 us).
 AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx) {
     const int n_tiles = (max_ctx + TKEYS - 1) / TKEYS;
-    const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;
+    const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;       // nw: slabs of the padded query tile (kernel instance)
     const int max_stages = hd >= 128 ? (nw > 4 ? 4 : 5) : 8;
-    const float t_tile = hd >= 128 ? 0.9f : (hd >= 64 ? 0.4f : 0.3f);
+    const float t_tile = hd >= 128 ? 2.0f : (hd >= 64 ? 1.3f : 0.8f);       // one iteration (ng tiles), measured
     AttnPlan best = {1, max_stages};
     float best_cost = 1e30f;
     const int depths[2] = {max_stages, max_stages >= 8 ? 4 : 3};
     for (int di = 0; di < 2; ++di) {
         const int stages = depths[di];
-        const int ng = (stages >= 4 && nw / n_slabs >= 2) ? 2 : 1;
+        const int ng = warp_groups(n_slabs, stages);
         for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
             int fit = fit_any(hd, nw, s, stages);
             if (fit <= 0) fit = std::max(1, 148 / s);               // no device to ask: assume one CTA per SM
             const int waves = (B * n_kv + fit - 1) / fit;
             const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
             const float stall = di == 0 ? 0.f : 0.25f * t_tile;      // a shallow ring hides less latency
-            const float cost = waves * (1.5f + iters * (t_tile + stall)) + (s > 1 ? 4.5f : 0.f);
+            const float cost = waves * (2.5f + iters * (t_tile + stall)) + (s > 1 ? 4.5f : 0.f);
             if (cost < best_cost - 1e-6f) { best_cost = cost; best = AttnPlan{s, stages}; }
         }
     }

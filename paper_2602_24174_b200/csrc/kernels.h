@@ -142,6 +142,7 @@ void launch_accept(const unsigned long long* argmax, const RowPlan& rp, const in
                    int32_t* n_accepted, int32_t* next_token, int32_t* target_tokens, long long* hist,
                    cudaStream_t stream);
 void launch_rope_table(float2* table, int max_positions, int hd, float base, cudaStream_t stream);
+void launch_wait_selftest(long long budget_cycles, int* status, cudaStream_t stream);
 // Teacher-forced targets built on the device from the drafts (see TASC_MODE_*).
 void launch_forced_targets(int mode, const int32_t* drafts, const int32_t* continuation, int64_t cont_stride,
                            const int32_t* len, const int32_t* prompt_len, int forced_accept, int vocab, int B, int k,

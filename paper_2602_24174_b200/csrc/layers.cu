@@ -275,6 +275,18 @@ __global__ void accept_kernel(const unsigned long long* __restrict__ argmax, Row
     if (hist) atomicAdd(reinterpret_cast<unsigned long long*>(hist + a), 1ull);
 }
 
+// Self-test of the bounded wait that every barrier wait of the tensor-core kernels goes through: waits on an
+// mbarrier that nothing will ever arrive at, for `budget` clock cycles, and records the outcome.
+__global__ void wait_selftest_kernel(long long budget, int* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+        if (!mbar_wait(smem_u32(&bar), 0, budget)) set_status(status, TASC_ETIMEOUT);
+        mbar_inval(smem_u32(&bar));
+    }
+}
+
 __global__ void rope_table_kernel(float2* table, int max_positions, int hd, float base) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int half = hd >> 1;
@@ -390,6 +402,10 @@ void launch_accept(const unsigned long long* argmax, const RowPlan& rp, const in
     ProfScope ps(K_ACCEPT, stream);
     accept_kernel<<<(B + 63) / 64, 64, 0, stream>>>(argmax, rp, drafts, forced_targets, tokens, stride, len, B, R,
                                                     n_accepted, next_token, target_tokens, hist);
+}
+void launch_wait_selftest(long long budget_cycles, int* status, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(budget_cycles, status);
 }
 void launch_rope_table(float2* table, int max_positions, int hd, float base, cudaStream_t stream) {
     ProfScope ps(K_OTHER, stream);

@@ -236,3 +236,20 @@ def test_config1_generate_graph_replay_equals_plain_enqueue(setup1):
         results.append((out.cpu().numpy(), st.steps, list(st.accepted_hist)))
     assert np.array_equal(results[0][0], results[1][0])
     assert results[0][1:] == results[1][1:]
+
+
+@pytest.mark.gpu
+def test_a_wait_that_nothing_ends_times_out_and_leaves_the_context_usable():
+    """The library's bounded barrier wait, driven to its limit on purpose by its own self-test kernel: the status word
+    reports the time-out, the kernel returns, and the device keeps working (no trap, no hang)."""
+    b = need_gpu()
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    b.tasc_selftest_bounded_wait(ws, 200_000)              # ~0.1 ms of SM cycles
+    with pytest.raises(b.TascError) as e:
+        b.tasc_poll_status(ws)
+    assert e.value.code == b.ETIMEOUT
+    b.tasc_poll_status(ws)                                 # cleared
+    x = torch.ones((8, 64), dtype=torch.bfloat16, device="cuda")
+    assert float(b.tasc_gemm_bf16(x, x).sum()) == 8 * 8 * 64
+    with pytest.raises(b.TascError):
+        b.tasc_selftest_bounded_wait(ws, 0)
