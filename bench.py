@@ -33,6 +33,20 @@ METRIC = "generated tokens/s with n-gram spec decode @1 B200; verify-step HBM GB
 UNIT = "tokens/s"
 
 
+# DRAM bytes per fused-GEMM launch from the ncu capture of the default workload (config 1, B=16, k=5), summarised in
+# profiles/gemm_fused_kernel_config1_b16_ncu.md: per layer 1.40 + 1.15 + 3.81 + 2.62 MB (QKV, O, gate/up, down) and
+# 28.4 MB for the LM head, over the step's 121 launches.  Valid for the kernel source whose digest is given;
+# any change of gemm_fused.cu makes the figure stale and `traffic` null.
+NCU_TRAFFIC = {"workload": (1, 16, 5), "bytes_per_launch": (30 * (1.404 + 1.149 + 3.812 + 2.624) * 1e6 + 28.4e6) / 121,
+               "kernel_sha256_16": "87db36a6624bf8ee"}
+
+
+def kernel_digest():
+    import hashlib
+    path = os.path.join(ROOT, "paper_2602_24174_b200", "csrc", "gemm_fused.cu")
+    return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -224,12 +238,26 @@ def main():
 
     # ---- inputs (seeded, synthetic); every rank is an independent replica with its own prompts
     host_w = W.make_weights(shape, cfg.seed_weights)
+    ctoks, coffs = corpus.make_corpus(cfg, n_docs=args.corpus_docs)
+    prompts_all = corpus.make_prompts(cfg, B * world)
+    if cfg.n_merged_tokens:
+        # configuration 3: merged n-gram tokens on top of the vocabulary (rows = constituent means), corpus and
+        # prompts re-tokenised by greedy longest match; selection from the first 20,000 documents
+        from dataclasses import replace
+        from workload import vocab_expand as VE
+        base = shape.vocab
+        sel = min(len(coffs) - 1, 20000)
+        merges = VE.select_merges(ctoks[:coffs[sel]], coffs[:sel + 1], cfg.n_merged_tokens, n_max=4, vocab=base)
+        host_w = VE.expand_weights(host_w, merges)
+        ctoks, coffs = VE.retokenize(ctoks, coffs, merges, vocab=base)
+        re = [VE.retokenize(pr, np.array([0, pr.size]), merges, vocab=base)[0] for pr in prompts_all]
+        plen = min(len(r) for r in re)
+        prompts_all = np.stack([r[:plen] for r in re]).astype(np.int32)
+        shape = replace(shape, vocab=base + len(merges))
     model = b.Model(shape, b.weights_to_device(host_w, shape.dtype, dev), max_positions=cfg.prompt_len + cfg.max_new + 4096,
                     page_size=cfg.page_size)
     del host_w
-    ctoks, coffs = corpus.make_corpus(cfg, n_docs=args.corpus_docs)
     drafter = b.tasc_drafter_build(torch.from_numpy(ctoks).to(dev), torch.from_numpy(coffs).to(dev), cfg.n_max, cfg.p_min, shape.vocab)
-    prompts_all = corpus.make_prompts(cfg, B * world)
     prompts = shard_prompts(prompts_all, rank, B)
     P = prompts.shape[1]
     total_steps = args.warmup + args.steps
@@ -328,7 +356,9 @@ def main():
     roofline = {
         "bound": "hbm", "kernel": "gemm_fused_kernel (tcgen05 + TMA, cluster split-K, fused epilogues; 4 launches per layer + LM head)",
         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-        "traffic": None, "peak_source": peaks["source"],
+        "traffic": (NCU_TRAFFIC["bytes_per_launch"] if (cfg.index, B, k) == NCU_TRAFFIC["workload"]
+                    and kernel_digest() == NCU_TRAFFIC["kernel_sha256_16"] else None),
+        "peak_source": peaks["source"],
         "bytes_per_launch_avg": gemm_bytes / max(gemm_launches, 1), "us_per_launch_avg": gemm_ms * 1e3 / max(gemm_launches, 1),
         "launches": gemm_launches,
         "verify_step": {"bytes_per_step": wbytes + kvbytes, "weight_bytes": wbytes, "kv_bytes": kvbytes,
@@ -394,8 +424,9 @@ def main():
             return {"tokens_per_s": B * max_new / (st.decode_ms * 1e-3), "decode_ms": st.decode_ms, "prefill_ms": st.prefill_ms,
                     "steps": st.steps, "mean_committed_per_step": st.committed / seq_steps, "accepted_hist": hist}
         gen["greedy"] = run_generate(b.MODE_GREEDY)
-        cont = torch.from_numpy(corpus.make_continuations(cfg, prompts, cfg.max_new + k + 1)).to(dev)
-        gen["teacher_forced_continuation"] = run_generate(b.MODE_CONTINUATION, cont=cont)
+        if not cfg.n_merged_tokens:          # held-out continuations are generated in the base vocabulary
+            cont = torch.from_numpy(corpus.make_continuations(cfg, prompts, cfg.max_new + k + 1)).to(dev)
+            gen["teacher_forced_continuation"] = run_generate(b.MODE_CONTINUATION, cont=cont)
         if args.sweep:
             gen["forced_accept_sweep"] = {str(a): run_generate(b.MODE_FORCED_ACCEPT, forced_accept=a) for a in range(k + 1)}
 
