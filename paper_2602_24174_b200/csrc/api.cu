@@ -77,8 +77,8 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     w.prompt_len = L.take<int32_t>(base, B);
     w.stop_len = L.take<int32_t>(base, B);
     w.x = L.take<float>(base, M * d.d_model);
-    // bf16: two rows per token plus tile padding (tiles of at most 128 tokens, rounded up to 16)
-    const size_t act_rows = d.dtype == TASC_F32 ? M : 2 * (M + 16 * (M / 128 + 1));
+    // (hi, lo) rows of every token tile, each tile padded to a multiple of 16 tokens (at most max(3, M / 128 + 1) tiles)
+    const size_t act_rows = d.dtype == TASC_F32 ? M : 2 * (M + 16 * (size_t)std::max<long long>(3, (long long)(M / 128 + 1)));
     w.h = L.take<uint8_t>(base, act_rows * d.d_model * esz);
     w.q = L.take<float>(base, M * m->q_dim);
     w.o = L.take<uint8_t>(base, act_rows * m->q_dim * esz);

@@ -218,7 +218,11 @@ tasc_status encode_tmap_kv(CUtensorMap* map, const void* ptr, uint64_t rows, int
 
 int gemm_token_tile(int M, bool pair) {
     const int cap = pair ? 128 : 256;                 // tokens per tile (UMMA N <= 256)
-    const int m_tiles = (M + cap - 1) / cap;
+    int m_tiles = (M + cap - 1) / cap;
+    // An MMA over a 128-row weight tile takes the same time for any number of token columns, while the split-K
+    // exchange, the accumulator read-out and the epilogue of a CTA grow with its columns: above 48 rows three
+    // (or more) token tiles per weight tile run faster than one or two wide ones (measured at 96, 192 and 448 rows).
+    if (pair && M > 48) m_tiles = std::max(m_tiles, 3);
     const int per = (M + m_tiles - 1) / m_tiles;
     return std::max(16, (per + 15) / 16 * 16);
 }
