@@ -228,9 +228,11 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     }
     if (lm_head) {
         const FusedPlan p_lm = plan_fused(M, d.vocab, d.d_model, EPI_LM);
+        CUtensorMap tm_h_lm;                       // the LM head's CTAs take several layout tiles at once
+        if ((st = encode_tmap_bf16(&tm_h_lm, w.h, rows, d.d_model, p_lm.BN)) != TASC_OK) return st;
         FusedArgs a = base;
         a.N = d.vocab; a.K = d.d_model; a.ssq_in = w.ssq; a.argmax = w.argmax; a.logits = logits;
-        if ((st = launch_gemm_fused(EPI_LM, &m->tm_lm, &tm_h, a, p_lm, s)) != TASC_OK) return st;
+        if ((st = launch_gemm_fused(EPI_LM, &m->tm_lm, &tm_h_lm, a, p_lm, s)) != TASC_OK) return st;
     }
     TASC_CUDA_TRY(cudaGetLastError());
     return TASC_OK;
@@ -533,7 +535,7 @@ extern "C" tasc_status tasc_gemm_bf16x2(const float* x, const void* wt, float* y
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + 256);
     const uint64_t rows = (uint64_t)p.m_tiles * p.BN;
     TASC_CUDA_TRY(cudaMemsetAsync(xs, 0, rows * K * 2, s));
-    launch_split_rows(x, xs, M, K, p.TB, s);
+    launch_split_rows(x, xs, M, K, p.TBL, s);
     CUtensorMap tmW, tmX;
     tasc_status st;
     if ((st = encode_tmap_bf16(&tmW, wt, N, K, 128)) != TASC_OK) return st;

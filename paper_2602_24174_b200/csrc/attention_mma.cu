@@ -198,26 +198,32 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
     }
     __syncthreads();
-    // TMA path (thread 0): a tile is four 16-token pages; each page of this KV head is one box (two for head_dim
-    // 128) of the [pages * kv_heads * 16][head_dim] view of the pool.  Rows past the key range re-read the range's
-    // last page and a page id outside the pool reads page 0: both are masked later, and nothing unmapped is touched.
-    auto load_tile_tma = [&](int tile, int stage) {
-        const uint32_t bar = smem_u32(&s_full[stage]);
-        const uint32_t kdst = smem_u32(Kt + stage * TILE_BYTES), vdst = smem_u32(Vt + stage * TILE_BYTES);
-        mbar_expect_tx(bar, 2u * TILE_BYTES);
-#pragma unroll
-        for (int pg = 0; pg < TKEYS / 16; ++pg) {
+    // TMA path (warp 0, one box per lane): a tile is four 16-token pages; each page of this KV head is one box (two
+    // for head_dim 128) of the [pages * kv_heads * 16][head_dim] view of the pool, for K and for V.  Rows past the
+    // key range re-read the range's last page and a page id outside the pool reads page 0: both are masked later,
+    // and nothing unmapped is touched.  A lane that issues one copy does not wait for the other lanes' copies, so
+    // the boxes of up to four tiles are requested in the time one thread needs for two.
+    constexpr int HB = HD == 128 ? 2 : 1;                      // 64-column boxes per row
+    constexpr int BOXES = (TKEYS / 16) * HB * 2;               // boxes of one tile: pages x halves x (K, V)
+    auto load_tiles_tma = [&](int sup) {
+        for (int idx = lane; idx < ng * BOXES; idx += 32) {
+            const int j = idx / BOXES, r = idx % BOXES;
+            const int tile = sup * ng + j;
+            if (tile >= n_tiles) continue;
+            const int stage = (sup % super_stages) * ng + j;
+            const int pg = r / (HB * 2), h = (r >> 1) % HB, is_v = r & 1;
+            const uint32_t bar = smem_u32(&s_full[stage]);
+            // the expected bytes may be posted after some of them have arrived: the phase cannot end before
+            // this arrival, which is the barrier's only one
+            if (r == 0) mbar_expect_tx(bar, 2u * TILE_BYTES);
             int key = k_begin + tile * TKEYS + pg * 16;
             key = key < k_end ? key : k_end - 1;
             int page = s_pages[key / 16 - pg_lo];
             page = page < 0 ? 0 : page;
             const int y = (page * a.n_kv + kh) * 16;
             constexpr int BOXB = (HD >= 64 ? 128 : 64) * 16;       // bytes of one box: 16 rows of at most 128 bytes
-#pragma unroll
-            for (int h = 0; h < (HD == 128 ? 2 : 1); ++h) {
-                tma_load_2d(kdst + h * (TKEYS * 128) + pg * BOXB, &tmK, h * 64, y, bar);
-                tma_load_2d(vdst + h * (TKEYS * 128) + pg * BOXB, &tmV, h * 64, y, bar);
-            }
+            const uint32_t dst = smem_u32((is_v ? Vt : Kt) + stage * TILE_BYTES) + h * (TKEYS * 128) + pg * BOXB;
+            tma_load_2d(dst, is_v ? &tmV : &tmK, h * 64, y, bar);
         }
     };
     // cp.async path: one row of the tile per TPR threads: a page lookup, then the thread's share of the row's chunks.
@@ -250,9 +256,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     };
     auto load_super = [&](int sup) {                             // the ng tiles of iteration `sup`
         if (use_tma) {
-            if (tid == 0)
-                for (int j = 0; j < ng; ++j)
-                    if (sup * ng + j < n_tiles) load_tile_tma(sup * ng + j, (sup % super_stages) * ng + j);
+            if (warp == 0) load_tiles_tma(sup);
         } else {
             for (int j = 0; j < ng; ++j)
                 if (sup * ng + j < n_tiles) load_tile(sup * ng + j, (sup % super_stages) * ng + j);
@@ -271,7 +275,6 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     log_at_exit.ta = global_ns();
 #endif
     griddep_launch_dependents();
-    for (; issued < super_stages - 1; ++issued) load_super(issued);   // commits an empty group past the end
 
     // Q rows of this KV head's group, scaled, as (hi, lo) bf16 in swizzled shared memory.  All global reads
     // are issued before the first conversion so that their latencies overlap.
@@ -286,6 +289,8 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (rho < G && rr < rows)
             qv[j] = *reinterpret_cast<const float4*>(a.q + (size_t)(b * R + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
     }
+    // the rest of the ring's prologue (tiles holding this step's new rows), requested while the Q rows are on their way
+    for (; issued < super_stages - 1; ++issued) load_super(issued);   // commits an empty group past the end
 #pragma unroll
     for (int j = 0; j < NQ; ++j) {
         const int i = tid + j * THREADS;

@@ -89,7 +89,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const uint32_t raw = smem_u32(smem_raw);
     uint8_t* smem = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
 
-    const int BN = a.BN, stages = a.stages, TB = a.TB;
+    const int BN = a.BN, stages = a.stages, TB = a.TB, TBL = a.TBL;   // TB tokens per CTA = one or more layout tiles of TBL
     const uint32_t b_stage_bytes = (uint32_t)BN * BK * 2;
     const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
     // [TB][128] this CTA's partial tile; behind the ring, except for the LM head, which has no cluster exchange
@@ -224,8 +224,8 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 *reinterpret_cast<float4*>(a.x + (size_t)m * a.N + f) = xv;
                 ss = xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w;
                 const float v[4] = {xv.x * gain4.x, xv.y * gain4.y, xv.z * gain4.z, xv.w * gain4.w};
-                const size_t row = (size_t)m_tile * (2 * TB) + t;
-                store_hilo4(a.a_out + row * a.N + f, a.a_out + (row + TB) * a.N + f, v);
+                const size_t row = (size_t)(m / TBL) * (2 * TBL) + m % TBL;
+                store_hilo4(a.a_out + row * a.N + f, a.a_out + (row + TBL) * a.N + f, v);
             }
             ss = warp_sum(ss);
             if (lane == 0) a.ssq_out[(size_t)m * a.ssq_out_slots + out_tile] = ss;
@@ -239,8 +239,8 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 float v[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) v[e] = gv[e] / (1.0f + expf(-gv[e])) * u[e];
-                const size_t row = (size_t)m_tile * (2 * TB) + t;
-                store_hilo4(a.a_out + row * a.N + j, a.a_out + (row + TB) * a.N + j, v);
+                const size_t row = (size_t)(m / TBL) * (2 * TBL) + m % TBL;
+                store_hilo4(a.a_out + row * a.N + j, a.a_out + (row + TBL) * a.N + j, v);
             }
         }
     };
@@ -265,15 +265,17 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             fence_barrier_init();
             tma_prefetch_desc(&tmW);
             tma_prefetch_desc(&tmX);
-            // The weights of the first stages depend on no earlier kernel: their loads start before the
-            // rest of the CTA is set up and before the preceding grid has finished.
-            for (int i = 0; i < pre; ++i) {
-                const uint32_t dstA = smem_u32(smem + (size_t)i * stage_bytes);
-                mbar_expect_tx_only(bar_full + 8u * i, A_STAGE_BYTES);
-                load_w(i, dstA, bar_full + 8u * i);
-            }
-            TL(1);
         }
+        __syncwarp();
+        // The weights of the first stages depend on no earlier kernel: their loads start before the rest of
+        // the CTA is set up and before the preceding grid has finished.  One lane per stage: a lane that has
+        // issued its copy does not wait for the others'.
+        if (lane < pre) {
+            const uint32_t dstA = smem_u32(smem + (size_t)lane * stage_bytes);
+            mbar_expect_tx_only(bar_full + 8u * lane, A_STAGE_BYTES);
+            load_w(lane, dstA, bar_full + 8u * lane);
+        }
+        if (lane == 0) TL(1);
         __syncwarp();
     } else if (warp == 5) {
         tmem_alloc(smem_u32(tmem_slot), ncols);
@@ -287,14 +289,15 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
+        griddep_wait();                 // every lane: the token rows below, and the epilogue operands later
+        if (lane < pre) {
+            const uint32_t dstB = smem_u32(smem + (size_t)lane * stage_bytes) + A_STAGE_BYTES;
+            mbar_expect_tx(bar_full + 8u * lane, b_stage_bytes);
+            tma_load_2d_hint(dstB, &tmX, (kb_begin + lane) * BK, m0, bar_full + 8u * lane, pol_x);
+        }
+        __syncwarp();
         if (lane == 0) {
-            griddep_wait();
             TL(2);
-            for (int i = 0; i < pre; ++i) {
-                const uint32_t dstB = smem_u32(smem + (size_t)i * stage_bytes) + A_STAGE_BYTES;
-                mbar_expect_tx(bar_full + 8u * i, b_stage_bytes);
-                tma_load_2d_hint(dstB, &tmX, (kb_begin + i) * BK, m0, bar_full + 8u * i, pol_x);
-            }
             for (int i = pre; i < n_kb; ++i) {
                 const int s = i % stages;
                 const uint32_t round = (uint32_t)(i / stages);
@@ -308,7 +311,6 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             TL(3);
         }
         __syncwarp();
-        griddep_wait();                 // every lane reads rows of earlier grids below
         late_prefetch();
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issue
@@ -368,32 +370,36 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         asm volatile("bar.sync 1, 128;" ::: "memory");          // s_inv visible to the four epilogue warps
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
         const int fl = warp * 32 + lane;                        // this thread's feature (TMEM lane) within the tile
-        for (int c = 0; c < TB; c += 32) {
-            const bool wide = c + 32 <= TB;                     // TB is a multiple of 16
-            uint32_t r[32];
-            if (have) {
-                if (wide) {
-                    uint32_t r2[32];
-                    tmem_ld32(lane_base + (uint32_t)c, r);
-                    tmem_ld32(lane_base + (uint32_t)(TB + c), r2);
-                    tmem_ld_wait();
+        // accumulator columns of layout tile lt: [lt * 2 TBL, +TBL) from the hi rows, the next TBL from the lo rows
+        for (int lt = 0; lt * TBL < TB; ++lt) {
+            const uint32_t col0 = (uint32_t)(lt * 2 * TBL);
+            for (int c = 0; c < TBL; c += 32) {
+                const bool wide = c + 32 <= TBL;                // TBL is a multiple of 16
+                uint32_t r[32];
+                if (have) {
+                    if (wide) {
+                        uint32_t r2[32];
+                        tmem_ld32(lane_base + col0 + (uint32_t)c, r);
+                        tmem_ld32(lane_base + col0 + (uint32_t)(TBL + c), r2);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                    } else {
+                        uint32_t q[16], q2[16];
+                        tmem_ld16(lane_base + col0 + (uint32_t)c, q);
+                        tmem_ld16(lane_base + col0 + (uint32_t)(TBL + c), q2);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(q[j]) + __uint_as_float(q2[j]));
+                    }
                 } else {
-                    uint32_t q[16], q2[16];
-                    tmem_ld16(lane_base + (uint32_t)c, q);
-                    tmem_ld16(lane_base + (uint32_t)(TB + c), q2);
-                    tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(q[j]) + __uint_as_float(q2[j]));
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
                 }
-            } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = 0u;
+                for (int j = 0; j < 32; ++j)
+                    if (j < 16 || wide) xch[(lt * TBL + c + j) * BM + fl] = __uint_as_float(r[j]);
             }
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (j < 16 || wide) xch[(c + j) * BM + fl] = __uint_as_float(r[j]);
         }
     }
     if (threadIdx.x == 0) TL(7);
@@ -456,13 +462,18 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             const float4 acc = *reinterpret_cast<const float4*>(xch + (size_t)t * BM + 4 * lane);
             const float v[4] = {acc.x, acc.y, acc.z, acc.w};
             const int f = f0 + 4 * lane;
-            unsigned long long best = 0ull;
+            // largest key of the warp's 128 features, then the smallest id that has it: two warp-wide reductions
+            uint32_t bk = 0u, bi = 0xFFFFFFFFu;
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                if (f + e < a.N) best = max(best, pack_argmax(v[e], (uint32_t)(f + e)));
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
-            if (lane == 0) atomicMax(&a.argmax[t0 + t], best);
+                if (f + e < a.N) {
+                    const uint32_t k = float_key(v[e]);
+                    if (bi == 0xFFFFFFFFu || k > bk) { bk = k; bi = (uint32_t)(f + e); }
+                }
+            const uint32_t mk = __reduce_max_sync(0xFFFFFFFFu, bk);
+            const uint32_t id = __reduce_min_sync(0xFFFFFFFFu, (bk == mk) ? bi : 0xFFFFFFFFu);
+            if (lane == 0 && id != 0xFFFFFFFFu)
+                atomicMax(&a.argmax[t0 + t], ((unsigned long long)mk << 32) | (unsigned long long)(0xFFFFFFFFu - id));
             if (a.logits) {
                 const float sc = s_inv[t];
 #pragma unroll
@@ -583,7 +594,11 @@ tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const Fus
 
 FusedPlan plan_fused(int M, int N, int K, int epi) {
     FusedPlan p;
-    p.TB = gemm_token_tile(M, true);
+    p.TBL = gemm_token_tile(M, true);
+    // The LM head streams the largest matrix once and has no split-K exchange: one CTA takes as many layout tiles
+    // as an MMA holds (256 columns), so that a weight tile is fetched by one CTA, not by one per token tile.
+    const int span = epi == EPI_LM ? std::max(1, std::min((M + p.TBL - 1) / p.TBL, 128 / p.TBL)) : 1;
+    p.TB = span * p.TBL;
     p.BN = 2 * p.TB;
     p.m_tiles = (M + p.TB - 1) / p.TB;
     p.out_tiles = epi == EPI_SWIGLU ? (N + 63) / 64 : (N + BM - 1) / BM;
@@ -631,7 +646,7 @@ FusedPlan plan_fused(int M, int N, int K, int epi) {
 tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
                               cudaStream_t stream) {
     if (a.M <= 0 || a.N <= 0 || a.K <= 0) return TASC_EINVAL;
-    a.num_kb = p.num_kb; a.BN = p.BN; a.TB = p.TB; a.stages = p.stages; a.pair = 1; a.data_bytes = p.data_bytes;
+    a.num_kb = p.num_kb; a.BN = p.BN; a.TB = p.TB; a.TBL = p.TBL; a.stages = p.stages; a.pair = 1; a.data_bytes = p.data_bytes;
     switch (epi) {
         case EPI_PLAIN:  return launch_epi<EPI_PLAIN>(tmW, tmX, a, p, K_GEMM, stream);
         case EPI_QKV:    return launch_epi<EPI_QKV>(tmW, tmX, a, p, K_GEMM, stream);

@@ -56,7 +56,7 @@ enum Epi {
 };
 struct FusedArgs {
     int M, N, K;                       // token rows, output features (EPI_SWIGLU: d_ff), reduction length
-    int num_kb, BN, TB, stages, pair, data_bytes;      // filled in by launch_gemm_fused from the plan
+    int num_kb, BN, TB, TBL, stages, pair, data_bytes; // filled in by launch_gemm_fused from the plan
     const float* ssq_in;               // [M][ssq_slots] partial sums of squares of the input rows (null: no scaling)
     int ssq_slots;
     float inv_d, eps;                  // rms factor = 1 / sqrt(sum(ssq) * inv_d + eps)
@@ -79,12 +79,13 @@ struct FusedArgs {
     int* status;
 };
 struct FusedPlan {
-    int TB, BN, m_tiles, out_tiles, num_kb;
+    int TBL;           // tokens per tile of the activation layout
+    int TB, BN, m_tiles, out_tiles, num_kb;   // TB: tokens per CTA (a multiple of TBL); BN = 2 TB; m_tiles: CTAs along the tokens
     int S;             // cluster size = k-splits
     int stages, data_bytes, smem_bytes;
 };
 FusedPlan plan_fused(int M, int N, int K, int epi);
-// tmW: weight map with box rows 128 (64 for EPI_SWIGLU); tmX: (hi, lo) activation map with box rows 2 TB.
+// tmW: weight map with box rows 128 (64 for EPI_SWIGLU); tmX: (hi, lo) activation map with box rows BN = 2 TB.
 tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
                               cudaStream_t stream);
 
