@@ -376,19 +376,40 @@ def main():
     h_next = torch.zeros(B, dtype=torch.int32).pin_memory()
     h_drafts = torch.zeros((B, k), dtype=torch.int32).pin_memory()
 
+    # the step itself is the same captured graph as in the device-resident timing (fresh buffers, so a fresh capture)
+    e2e_graph = None
+    if not args.no_graph:
+        for _ in range(2):
+            one_step(kvs, seqs, tokens, length)
+        cap_stream = torch.cuda.Stream(device=dev)
+        cap_stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cap_stream):
+            e2e_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(e2e_graph, stream=cap_stream):
+                e2e_out = one_step(kvs, seqs, tokens, length)
+        torch.cuda.current_stream().wait_stream(cap_stream)
+        torch.cuda.synchronize()
+    np_tokens, np_len = h_tokens.numpy(), h_len.numpy()        # views of the pinned buffers
+    np_acc, np_next, np_drafts = h_acc.numpy(), h_next.numpy(), h_drafts.numpy()
+    rows_idx = np.arange(B)
+
     def e2e_step():
         tokens.copy_(h_tokens, non_blocking=True)
         length.copy_(h_len, non_blocking=True)
-        n_acc, nxt, _, _ = one_step(kvs, seqs, tokens, length)
+        if e2e_graph is not None:
+            e2e_graph.replay()
+            n_acc, nxt = e2e_out[0], e2e_out[1]
+        else:
+            n_acc, nxt, _, _ = one_step(kvs, seqs, tokens, length)
         h_acc.copy_(n_acc, non_blocking=True)
         h_next.copy_(nxt, non_blocking=True)
         h_drafts.copy_(drafts, non_blocking=True)
-        torch.cuda.synchronize()
-        for i in range(B):                       # host-side commit of the step's result
-            L, a = int(h_len[i]), int(h_acc[i])
-            h_tokens[i, L:L + a] = h_drafts[i, :a]
-            h_tokens[i, L + a] = h_next[i]
-            h_len[i] = L + a + 1
+        torch.cuda.current_stream().synchronize()
+        for j in range(k):                       # host-side commit of the step's result: accepted drafts, then the next token
+            sel = np_acc > j
+            np_tokens[rows_idx[sel], np_len[sel] + j] = np_drafts[sel, j]
+        np_tokens[rows_idx, np_len + np_acc] = np_next
+        np.add(np_len, np_acc + 1, out=np_len)
 
     for _ in range(args.warmup):
         e2e_step()
