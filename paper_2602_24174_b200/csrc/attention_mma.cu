@@ -653,10 +653,15 @@ int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
 // cluster occupancy dictates (one straggling cluster costs a whole wave), and splitting adds the cluster
 // exchange and merge (about 4.5 us).
 AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx) {
-    const int n_tiles = (max_ctx + TKEYS - 1) / TKEYS;
+    // The launch shape is fixed before the lengths are known (and stays fixed in a captured graph): it is chosen
+    // for three quarters of the context the cache can hold; shorter ranges leave the last splits idle.
+    const int n_tiles = std::max(1, ((max_ctx * 3) / 4 + TKEYS - 1) / TKEYS);
     const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;       // nw: slabs of the padded query tile (kernel instance)
     const int max_stages = hd >= 128 ? (nw > 4 ? 4 : 5) : 8;
-    const float t_tile = hd >= 128 ? 2.0f : (hd >= 64 ? 1.3f : 0.8f);       // one iteration (ng tiles), measured
+    // Measured (microseconds): one iteration of a warp group over a 64-key tile, and the time the SM's mma.sync
+    // pipes need per tile and 16-row slab when all warps have work (the lower bound once several groups run).
+    const float t_tile = hd >= 128 ? 2.0f : (hd >= 64 ? 1.3f : 0.8f);
+    const float t_pipe = hd >= 128 ? 0.6f : (hd >= 64 ? 0.3f : 0.15f);
     AttnPlan best = {1, max_stages};
     float best_cost = 1e30f;
     const int depths[2] = {max_stages, max_stages >= 8 ? 4 : 3};
@@ -667,9 +672,14 @@ AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx) {
             int fit = fit_any(hd, nw, s, stages);
             if (fit <= 0) fit = std::max(1, 148 / s);               // no device to ask: assume one CTA per SM
             const int waves = (B * n_kv + fit - 1) / fit;
-            const int iters = ((n_tiles + s - 1) / s + ng - 1) / ng;
+            const int tiles_cta = (n_tiles + s - 1) / s;
+            const int iters = (tiles_cta + ng - 1) / ng;
             const float stall = di == 0 ? 0.f : 0.25f * t_tile;      // a shallow ring hides less latency
-            const float cost = waves * (2.5f + iters * (t_tile + stall)) + (s > 1 ? 4.5f : 0.f);
+            const float loop = std::max(iters * (t_tile + stall), tiles_cta * n_slabs * t_pipe);
+            const float merge = s > 1 ? 0.5f + 0.25f * s : 0.f;      // cluster barrier + one round of remote reads
+            // a grid that takes (nearly) every SM keeps the next kernel's CTAs from starting early
+            const float crowd = B * n_kv * s > 128 ? 3.0f : 0.f;
+            const float cost = waves * (2.5f + loop) + merge + crowd;
             if (cost < best_cost - 1e-6f) { best_cost = cost; best = AttnPlan{s, stages}; }
         }
     }
