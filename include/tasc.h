@@ -163,13 +163,16 @@ typedef struct {
 tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc_weights* weights, tasc_model** out);
 tasc_status tasc_model_destroy(tasc_model* m);
 
-/* Bytes of workspace that step calls need for up to B_max sequences and k_max drafts. */
+/* Bytes of workspace that step calls need for up to B_max sequences and k_max drafts.  bf16 models reserve
+ * room for at least 1,024 rows in flight, which prefill passes of few sequences use (tens of MB at most). */
 size_t tasc_workspace_bytes(const tasc_model* m, int32_t B_max, int32_t k_max);
 
 /*
  * Run the committed tokens 0 .. len[b]-2 of every sequence through the model to fill the KV
- * cache (no logits).  max_len (host value) >= every len[b]; it fixes the number of chunks.
- * Asynchronous.  Errors: EINVAL.
+ * cache (no logits).  max_len (host value) >= every len[b]; it fixes the number of passes: a pass
+ * carries 16 positions of every sequence (float32 models) or as many as the workspace holds, up to 256
+ * per sequence (bf16 models), through the same kernels as a verify step; sequences shorter than a
+ * pass's range take no part in it.  Asynchronous.  Errors: EINVAL.
  */
 tasc_status tasc_prefill(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, int32_t B, int32_t max_len,
                          void* workspace, size_t workspace_bytes, tasc_stream stream);

@@ -54,11 +54,26 @@ struct Workspace {
     size_t bytes;
 };
 
-// The layout is always made for TASC_MAX_ROWS rows per sequence so that every call agrees on it.
+// Rows a pass may carry: TASC_MAX_ROWS per sequence for a verify step, and for bf16 models at least PREFILL_ROWS
+// in all, so that a prefill of few sequences still runs passes of hundreds of rows (weights are read once per pass).
+constexpr int PREFILL_ROWS = 1024;
+constexpr int PREFILL_ROWS_PER_SEQ = 256;
+size_t workspace_rows(const tasc_model* m, int B) {
+    const size_t verify = (size_t)B * TASC_MAX_ROWS;
+    return m->desc.dtype == TASC_F32 ? verify : std::max<size_t>(verify, PREFILL_ROWS);
+}
+// Rows per sequence of one prefill pass: a multiple of 16 that fits the workspace.
+int prefill_rows(const tasc_model* m, int B) {
+    if (m->desc.dtype == TASC_F32) return TASC_MAX_ROWS;
+    const int per = (int)(workspace_rows(m, B) / (size_t)B) / 16 * 16;
+    return std::max(TASC_MAX_ROWS, std::min(per, PREFILL_ROWS_PER_SEQ));
+}
+
+// The layout is always made for workspace_rows() rows so that every call agrees on it.
 Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     const tasc_model_desc& d = m->desc;
     uint8_t* base = static_cast<uint8_t*>(base_);
-    const size_t M = (size_t)B * TASC_MAX_ROWS;
+    const size_t M = workspace_rows(m, B);
     const size_t esz = d.dtype == TASC_F32 ? 4 : 2;
     Layout L;
     Workspace w;
@@ -172,7 +187,10 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
-    const AttnPlan att_plan = plan_attention_mma(B, d.n_kv_heads, d.head_dim, (d.n_q_heads / d.n_kv_heads) * R, max_ctx);
+    // attention works on blocks of at most 16 rows per sequence (one block in a verify step, several in a prefill pass)
+    const int att_rows = R <= 16 ? R : 16;
+    const AttnPlan att_plan = plan_attention_mma(B * (R / att_rows), d.n_kv_heads, d.head_dim,
+                                                 (d.n_q_heads / d.n_kv_heads) * att_rows, max_ctx);
     const int TB = gemm_token_tile(M, true);
     const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
     CUtensorMap tm_h, tm_o, tm_act;
@@ -266,7 +284,7 @@ tasc_status verify_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_se
 
 tasc_status prefill_enqueue(const tasc_model* m, const tasc_kv* kv, const tasc_seqs* seqs, const Workspace& w, int B,
                             int max_len, cudaStream_t s) {
-    const int R = TASC_MAX_ROWS;
+    const int R = prefill_rows(m, B);
     const int chunks = (std::max(max_len - 1, 0) + R - 1) / R;
     for (int c = 0; c < chunks; ++c) {
         tasc_status st = forward_any(m, kv, w, RowSource{seqs, nullptr, c}, B, R, false, nullptr, s);

@@ -42,7 +42,8 @@ struct AttnArgs {
     const int* seq_rows;
     __nv_bfloat16* out;                // (hi, lo) activation buffer, row length n_q * hd
     int TB;
-    int R, n_q, n_kv, splits, stages;
+    int R, n_q, n_kv, splits, stages;  // R: rows per sequence in this pass
+    int Rs, n_sub;                     // a CTA takes Rs of them (sub-block blockIdx.z % n_sub); R = Rs * n_sub
     int use_tma;                       // K/V tiles by TMA box loads (16-token pages); otherwise by cp.async
     int* status;
     float scale_log2e;
@@ -134,19 +135,23 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     __shared__ int s_pages[MAX_STAGED_PAGES];
     __shared__ uint64_t s_full[8];               // one per ring stage: bytes of its K and V tile have landed (TMA path)
 
-    const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z;
+    const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z / a.n_sub, rb = (blockIdx.z % a.n_sub) * a.Rs;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef TASC_TIMELINE
     struct LogAtExit { unsigned long long t0, ta, tb, tc, td, te, tf; __device__ ~LogAtExit() { if (threadIdx.x == 0) ctalog_put(t0, ta, tb, 10, tc, td, te, tf); } } log_at_exit{global_ns(), 0, 0, 0, 0, 0, 0};
 #endif
-    const int g = a.n_q / a.n_kv, R = a.R;
+    const int g = a.n_q / a.n_kv, R = a.Rs;                   // R: rows of this CTA's sub-block; its first row is rb
     const int G = g * R;
     const int qd = a.n_q * HD;
 
     // The row plan, the block table and the K/V of committed positions were written before the
     // preceding grid started, so they may be read ahead of griddepcontrol.wait.
-    const int rows = a.seq_rows[b];
-    const int pos0 = a.seq_pos0[b];
+    // A pass with more than Rs rows per sequence (prefill) is cut into sub-blocks of Rs rows; the rows before this
+    // sub-block are ordinary keys to it, but they were written by the preceding grid like its own.
+    const int seq_pos0 = a.seq_pos0[b];                        // committed positions: in the cache before this pass
+    int rows = a.seq_rows[b] - rb;
+    rows = rows < 0 ? 0 : (rows > R ? R : rows);
+    const int pos0 = seq_pos0 + rb;
     if (rows == 0) {
         griddep_wait();
         griddep_launch_dependents();
@@ -154,7 +159,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (sp == 0) {
             for (int i = tid; i < G * (HD / 4); i += THREADS) {
                 const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
-                const int m = b * R + rho % R;
+                const int m = b * a.R + rb + rho % R;
                 const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
                 const size_t col = (size_t)(kh * g + rho / R) * HD + d4;
                 *reinterpret_cast<uint2*>(a.out + row * qd + col) = make_uint2(0u, 0u);
@@ -266,7 +271,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // prologue of the ring: tiles that lie wholly inside the committed prefix start before the wait,
     // the tiles holding this step's new rows (written by the preceding grid) after it
     int issued = 0;
-    while (issued < super_stages - 1 && issued < n_super && k_begin + (issued + 1) * ng * TKEYS <= pos0) {
+    while (issued < super_stages - 1 && issued < n_super && k_begin + (issued + 1) * ng * TKEYS <= seq_pos0) {
         load_super(issued);
         ++issued;
     }
@@ -287,7 +292,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int hl = rho / R, rr = rho % R;
         qv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rho < G && rr < rows)
-            qv[j] = *reinterpret_cast<const float4*>(a.q + (size_t)(b * R + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
+            qv[j] = *reinterpret_cast<const float4*>(a.q + (size_t)(b * a.R + rb + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
     }
     // the rest of the ring's prologue (tiles holding this step's new rows), requested while the Q rows are on their way
     for (; issued < super_stages - 1; ++issued) load_super(issued);   // commits an empty group past the end
@@ -475,7 +480,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (rho >= G) continue;
                 const int hl = rho / R, rr = rho % R;
                 const float inv = (rr < rows) ? (half ? inv1 : inv0) : 0.f;
-                const int m = b * R + rr;
+                const int m = b * a.R + rb + rr;
                 const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
                 const size_t col = (size_t)(kh * g + hl) * HD + 2 * (lane & 3);
 #pragma unroll
@@ -546,7 +551,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const float inv = den > 0.f ? 1.0f / den : 0.f;
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
         }
-        const int m = b * R + rr;
+        const int m = b * a.R + rb + rr;
         const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
         const size_t col = (size_t)(kh * g + hl) * HD + d4;
         uint2 h, l;
@@ -691,7 +696,11 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
                                  const AttnPlan& plan, int* status, cudaStream_t stream) {
     const int n_splits = plan.splits;
-    const int G = (n_q / n_kv) * R;
+    // up to 16 rows per sequence (a verify step) are one block; longer passes (prefill) are cut into blocks of 16
+    const int Rs = R <= 16 ? R : 16;
+    if (R % Rs) return TASC_EINVAL;
+    const int n_sub = R / Rs;
+    const int G = (n_q / n_kv) * Rs;
     if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 8) return TASC_EINVAL;
     const int GP = attention_mma_row_pad(G);
     AttnArgs a;
@@ -699,7 +708,7 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
     a.max_pages = max_pages; a.page_size = page_size; a.n_pages = n_pages;
     a.seq_pos0 = rp.seq_pos0; a.seq_rows = rp.seq_rows;
     a.out = out; a.TB = TB;
-    a.R = R; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits; a.stages = plan.stages;
+    a.R = R; a.Rs = Rs; a.n_sub = n_sub; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits; a.stages = plan.stages;
     a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
     a.status = status;
     // 16-token pages arrive as TMA boxes; any other page size takes the cp.async path of the same kernel
@@ -714,13 +723,13 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
         if ((st = encode_tmap_kv(&tmV, v_pages, rows, hd)) != TASC_OK) return st;
     }
     if (GP == 64) {
-        if (hd == 32) return launch_inst<32, 4>(a, tmK, tmV, B, stream);
-        if (hd == 64) return launch_inst<64, 4>(a, tmK, tmV, B, stream);
-        return launch_inst<128, 4>(a, tmK, tmV, B, stream);
+        if (hd == 32) return launch_inst<32, 4>(a, tmK, tmV, B * n_sub, stream);
+        if (hd == 64) return launch_inst<64, 4>(a, tmK, tmV, B * n_sub, stream);
+        return launch_inst<128, 4>(a, tmK, tmV, B * n_sub, stream);
     }
-    if (hd == 32) return launch_inst<32, 8>(a, tmK, tmV, B, stream);
-    if (hd == 64) return launch_inst<64, 8>(a, tmK, tmV, B, stream);
-    return launch_inst<128, 8>(a, tmK, tmV, B, stream);
+    if (hd == 32) return launch_inst<32, 8>(a, tmK, tmV, B * n_sub, stream);
+    if (hd == 64) return launch_inst<64, 8>(a, tmK, tmV, B * n_sub, stream);
+    return launch_inst<128, 8>(a, tmK, tmV, B * n_sub, stream);
 }
 
 }  // namespace tasc

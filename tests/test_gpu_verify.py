@@ -201,6 +201,43 @@ def test_config4_shape_long_context_lockstep():
 
 
 @pytest.mark.gpu
+def test_bf16_prefill_of_ragged_lengths_in_wide_passes():
+    """Prompts of 300, 37, 129 and 257 tokens in one batch of configuration 1's geometry (two layers): the bf16
+    prefill runs passes of 256 rows per sequence, cut into blocks of 16 rows for the attention, so the batch has
+    a sequence that needs a second pass, sequences that end inside a block, and one whose second pass is a single
+    row.  The verify step that follows must see the cache the oracle builds token by token."""
+    b = need_gpu()
+    cfg = configs.shrunk(configs.get(1), n_layers=2, n_docs=2000)
+    s = make_setup(cfg, build_drafter=False, oracle_ngrams=False)
+    lens = [300, 37, 129, 257]
+    B, k = len(lens), cfg.k
+    rng = np.random.default_rng(5)
+    stride = max(lens) + 4 * (k + 1)
+    host = np.zeros((B, stride), dtype=np.int32)
+    for i, L in enumerate(lens):
+        host[i, :L] = rng.integers(0, cfg.model.vocab, L)
+    drafts_h = rng.integers(0, cfg.model.vocab, (B, k)).astype(np.int32)
+    tokens = torch.from_numpy(host).cuda()
+    length = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    pool, bt, kv = s.model.new_kv(B, stride + b.MAX_ROWS)
+    ws = s.model.new_workspace(B, k)
+    seqs = b.make_seqs(tokens, length)
+    b.tasc_prefill(s.model, kv, seqs, B, max(lens), ws)
+    n_acc, nxt, tgt, logits = b.tasc_verify_step(s.model, kv, seqs, torch.from_numpy(drafts_h).cuda(), ws,
+                                                 want_targets=True, want_logits=True)
+    b.tasc_poll_status(ws)
+    lg, tgt = logits.cpu().numpy(), tgt.cpu().numpy()
+    for i, L in enumerate(lens):
+        cache = s.oracle.new_cache(L + k + 1)
+        s.oracle.prefill(host[i, :L - 1], cache)
+        st = G.verify_step(s.oracle, cache, int(host[i, L - 1]), list(map(int, drafts_h[i])), keep_logits=True)
+        err = np.abs(lg[i] - st.logits)
+        assert (err <= BF16_TOL["logit_atol"] + BF16_TOL["logit_rtol"] * np.abs(st.logits)).all(), (i, float(err.max()))
+        for r in range(k + 1):
+            assert int(tgt[i, r]) == st.y[r] or st.gap[r] < BF16_TOL["gap_tol"], (i, r)
+
+
+@pytest.mark.gpu
 def test_config2_batch32_k3_and_k8_one_step():
     """Batch 32 of configuration 2's geometry at k = 3 (M = 128 rows, one token tile) and k = 8 (M = 288 rows, three
     token tiles of 96), two layers."""
