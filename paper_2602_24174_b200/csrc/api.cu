@@ -224,6 +224,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
         a.k_pages = static_cast<__nv_bfloat16*>(kvl.k); a.v_pages = static_cast<__nv_bfloat16*>(kvl.v);
         a.block_table = kv->block_table; a.max_pages = kv->max_pages_per_seq; a.page_size = d.page_size; a.n_pages = kv->n_pages;
         a.R = R; a.n_q = d.n_q_heads; a.n_kv = d.n_kv_heads; a.hd = d.head_dim; a.max_positions = d.max_positions;
+        a.early = l > 0;               // layer 0 follows the kernel that writes the row plan
         if ((st = launch_gemm_fused(EPI_QKV, &m->tm_qkv[l], &tm_h, a, p_qkv, s)) != TASC_OK) return st;
 
         st = launch_attention_mma(w.q, static_cast<const __nv_bfloat16*>(kvl.k), static_cast<const __nv_bfloat16*>(kvl.v),
@@ -233,6 +234,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
 
         a = base;
         a.N = d.d_model; a.K = m->q_dim; a.x = w.x; a.gain = m->mlp_norm[l]; a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = w.ssq_slots;
+        a.early = 1;                   // x was last written three launches back
         if ((st = launch_gemm_fused(EPI_RESID, &m->tm_o[l], &tm_o, a, p_o, s)) != TASC_OK) return st;
 
         a = base;
@@ -242,6 +244,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
         a = base;
         a.N = d.d_model; a.K = d.d_ff; a.x = w.x; a.gain = l + 1 < d.n_layers ? m->attn_norm[l + 1] : m->final_norm;
         a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = w.ssq_slots;
+        a.early = 1;                   // x was last written two launches back
         if ((st = launch_gemm_fused(EPI_RESID, &m->tm_down[l], &tm_act, a, p_down, s)) != TASC_OK) return st;
     }
     if (lm_head) {

@@ -245,7 +245,10 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
     };
     Pre pf[NPF];
-    auto late_prefetch = [&]() {                // warps 4 and 5, after their producer / MMA loops
+    // Where the epilogue's operands were complete before the preceding grid began (a.early: the row plan, rotary
+    // table and page ids of a QKV launch that does not follow the row-plan kernel; the residual rows and gain of a
+    // RESID launch), they are requested ahead of griddepcontrol.wait, otherwise after it.
+    auto late_prefetch = [&]() {
         if (EPI != EPI_LM) {
 #pragma unroll
             for (int i = 0; i < NPF; ++i)
@@ -289,6 +292,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
+        if (a.early) late_prefetch();
         griddep_wait();                 // every lane: the token rows below, and the epilogue operands later
         if (lane < pre) {
             const uint32_t dstB = smem_u32(smem + (size_t)lane * stage_bytes) + A_STAGE_BYTES;
@@ -311,9 +315,10 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             TL(3);
         }
         __syncwarp();
-        late_prefetch();
+        if (!a.early) late_prefetch();
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issue
+        if (a.early) late_prefetch();
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
             bool ok = true;
@@ -338,19 +343,15 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
         __syncwarp();
         griddep_wait();
-        late_prefetch();
+        if (!a.early) late_prefetch();
     } else {
         // ------------------------------------------------------------ epilogue, part 1: accumulator -> shared memory
+        if (a.early) late_prefetch();
         griddep_wait();
 #ifdef TASC_TIMELINE
         if (threadIdx.x == 0) g_ta = global_ns();
 #endif
-        if (EPI != EPI_LM) {
-#pragma unroll
-            for (int i = 0; i < NPF; ++i)
-                if (warp + EW * i < count) pf[i] = prefetch(warp + EW * i);
-            if (EPI == EPI_RESID && f0 + 4 * lane < a.N) gain4 = *reinterpret_cast<const float4*>(a.gain + f0 + 4 * lane);
-        }
+        if (!a.early) late_prefetch();
         if (EPI == EPI_QKV || EPI == EPI_SWIGLU || EPI == EPI_LM || (EPI == EPI_PLAIN && a.ssq_in)) {
             for (int t = threadIdx.x; t < TB; t += 128) {
                 const int m = t0 + t;

@@ -57,6 +57,7 @@ enum Epi {
 struct FusedArgs {
     int M, N, K;                       // token rows, output features (EPI_SWIGLU: d_ff), reduction length
     int num_kb, BN, TB, TBL, stages, pair, data_bytes; // filled in by launch_gemm_fused from the plan
+    int early;                         // the epilogue's global operands were complete before the preceding grid began
     const float* ssq_in;               // [M][ssq_slots] partial sums of squares of the input rows (null: no scaling)
     int ssq_slots;
     float inv_d, eps;                  // rms factor = 1 / sqrt(sum(ssq) * inv_d + eps)
