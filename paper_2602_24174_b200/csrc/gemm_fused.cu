@@ -231,16 +231,24 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             if (lane == 0) a.ssq_out[(size_t)m * a.ssq_out_slots + out_tile] = ss;
         } else if (EPI == EPI_SWIGLU) {
             const float sc = s_inv[t];
-            const float4 up = shfl_xor4(acc, 16);              // lanes 0-15 hold gate features, 16-31 the up features
-            const int j = f0 + 4 * lane;
-            if (lane < 16 && j < a.N) {
-                const float gv[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
-                const float u[4] = {up.x * sc, up.y * sc, up.z * sc, up.w * sc};
-                float v[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) v[e] = gv[e] / (1.0f + expf(-gv[e])) * u[e];
+            // lanes 0-15 hold four gate features each, lanes 16-31 the matching up features: after the exchange both
+            // lanes of a pair have all eight values, and each finishes two of the four outputs
+            const float4 oth = shfl_xor4(acc, 16);
+            const bool low = lane < 16;
+            const float4 g4 = low ? acc : oth, u4 = low ? oth : acc;
+            const int j = f0 + 4 * (lane & 15) + (low ? 0 : 2);
+            if (j < a.N) {                                       // d_ff is a multiple of 8: j + 1 < N as well
+                const float g0 = (low ? g4.x : g4.z) * sc, g1 = (low ? g4.y : g4.w) * sc;
+                const float u0 = (low ? u4.x : u4.z) * sc, u1 = (low ? u4.y : u4.w) * sc;
+                const float v0 = g0 / (1.0f + expf(-g0)) * u0, v1 = g1 / (1.0f + expf(-g1)) * u1;
+                __nv_bfloat16 h0, l0, h1, l1;
+                split_bf16(v0, h0, l0);
+                split_bf16(v1, h1, l1);
                 const size_t row = (size_t)(m / TBL) * (2 * TBL) + m % TBL;
-                store_hilo4(a.a_out + row * a.N + j, a.a_out + (row + TBL) * a.N + j, v);
+                *reinterpret_cast<uint32_t*>(a.a_out + row * a.N + j) =
+                    (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                *reinterpret_cast<uint32_t*>(a.a_out + (row + TBL) * a.N + j) =
+                    (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
             }
         }
     };
@@ -459,27 +467,46 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     } else {
         // LM head: per token row the largest logit of this 128-feature tile (smallest id on ties), merged
         // across tiles by an atomic max on the packed (value, id) word; the logits themselves are not stored
-        for (int t = warp; t < valid; t += EW) {
-            const float4 acc = *reinterpret_cast<const float4*>(xch + (size_t)t * BM + 4 * lane);
-            const float v[4] = {acc.x, acc.y, acc.z, acc.w};
-            const int f = f0 + 4 * lane;
-            // largest key of the warp's 128 features, then the smallest id that has it: two warp-wide reductions
-            uint32_t bk = 0u, bi = 0xFFFFFFFFu;
+        // (two token rows per round: their reductions are independent and overlap)
+        const int f = f0 + 4 * lane;
+        for (int tb = warp; tb < valid; tb += 2 * EW) {
+            float4 acc[2];
+            uint32_t bk[2], bi[2];
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (f + e < a.N) {
-                    const uint32_t k = float_key(v[e]);
-                    if (bi == 0xFFFFFFFFu || k > bk) { bk = k; bi = (uint32_t)(f + e); }
-                }
-            const uint32_t mk = __reduce_max_sync(0xFFFFFFFFu, bk);
-            const uint32_t id = __reduce_min_sync(0xFFFFFFFFu, (bk == mk) ? bi : 0xFFFFFFFFu);
-            if (lane == 0 && id != 0xFFFFFFFFu)
-                atomicMax(&a.argmax[t0 + t], ((unsigned long long)mk << 32) | (unsigned long long)(0xFFFFFFFFu - id));
-            if (a.logits) {
-                const float sc = s_inv[t];
+            for (int u = 0; u < 2; ++u) {
+                const int t = tb + u * EW;
+                acc[u] = t < valid ? *reinterpret_cast<const float4*>(xch + (size_t)t * BM + 4 * lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const float v[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
+                // largest key of the warp's 128 features, then the smallest id that has it: two warp-wide reductions
+                bk[u] = 0u; bi[u] = 0xFFFFFFFFu;
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (f + e < a.N) a.logits[(size_t)(t0 + t) * a.N + f + e] = v[e] * sc;
+                    if (f + e < a.N) {
+                        const uint32_t k = float_key(v[e]);
+                        if (bi[u] == 0xFFFFFFFFu || k > bk[u]) { bk[u] = k; bi[u] = (uint32_t)(f + e); }
+                    }
+            }
+            uint32_t mk[2], id[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) mk[u] = __reduce_max_sync(0xFFFFFFFFu, bk[u]);
+#pragma unroll
+            for (int u = 0; u < 2; ++u) id[u] = __reduce_min_sync(0xFFFFFFFFu, (bk[u] == mk[u]) ? bi[u] : 0xFFFFFFFFu);
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int t = tb + u * EW;
+                if (t >= valid) continue;
+                if (lane == 0 && id[u] != 0xFFFFFFFFu)
+                    atomicMax(&a.argmax[t0 + t], ((unsigned long long)mk[u] << 32) | (unsigned long long)(0xFFFFFFFFu - id[u]));
+                if (a.logits) {
+                    const float sc = s_inv[t];
+                    const float v[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (f + e < a.N) a.logits[(size_t)(t0 + t) * a.N + f + e] = v[e] * sc;
+                }
             }
         }
     }
