@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # profiles/gemm_fused_kernel_config1_b16_ncu.md: per layer 1.40 + 1.15 + 3.81 + 2.62 MB (QKV, O, gate/up, down) and
 # 28.4 MB for the LM head, over the step's 121 launches.  Valid for the kernel source whose digest is given;
 # any change of gemm_fused.cu makes the figure stale and `traffic` null.
-NCU_TRAFFIC = {"workload": (1, 16, 5), "bytes_per_launch": (30 * (1.418 + 1.151 + 3.811 + 2.625) * 1e6 + 56.88e6) / 121,
-               "kernel_sha256_16": "4aedbe729bdf07be"}
+NCU_TRAFFIC = {"workload": (1, 16, 5), "bytes_per_launch": (30 * (1.418 + 1.151 + 3.807 + 2.625) * 1e6 + 56.88e6) / 121,
+               "kernel_sha256_16": "f52e0421899d7888"}
 
 
 def kernel_digest():
