@@ -251,6 +251,7 @@ draft_kernel(const DeviceTables dt, const int32_t* __restrict__ tokens, int64_t 
     extern __shared__ int32_t dsm[];
     int32_t* h_tok = dsm;                                          // [hs] token or -1
     uint32_t* h_cnt = reinterpret_cast<uint32_t*>(dsm + hs_mask + 1);   // [hs] count, bit 31 = seen in the corpus list
+    int32_t* s_seq = dsm + 2 * (hs_mask + 1);                      // [L] the committed tokens: every draft scans them twice
     __shared__ Best red[DRAFT_THREADS / 32];
     __shared__ int s_suffix[TASC_MAX_ORDER];     // last n_max tokens of the query, newest last
     __shared__ int s_nstar, s_tprompt;
@@ -259,12 +260,14 @@ draft_kernel(const DeviceTables dt, const int32_t* __restrict__ tokens, int64_t 
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int32_t* seq = tokens + (int64_t)b * stride;
     int L = len[b];
     L = L < 0 ? 0 : (L > stride ? (int)stride : L);
     const int n_max = dt.n_max;
     const bool use_corp = lam_num > 0, use_prompt = lam_num < lam_den;
 
+    for (int i = tid; i < L; i += DRAFT_THREADS) s_seq[i] = tokens[(int64_t)b * stride + i];
+    __syncthreads();
+    const int32_t* seq = s_seq;
     if (tid < TASC_MAX_ORDER) {
         const int p = L - n_max + tid;             // suffix slot tid <-> position p (only the last n_max slots are used)
         s_suffix[tid] = (tid < n_max && p >= 0) ? seq[p] : -1;
@@ -572,10 +575,10 @@ extern "C" tasc_status tasc_draft(const tasc_drafter* d, const int32_t* tokens, 
         return TASC_EINVAL;
     uint64_t hs = 64;
     while (hs * 3 < (uint64_t)stride * 4) hs <<= 1;      // load factor <= 3/4
-    const size_t smem = hs * 8;
+    const size_t smem = hs * 8 + (size_t)stride * sizeof(int32_t);      // hash of the context successors + the tokens
     static bool attr = false;
     if (!attr) {
-        TASC_CUDA_TRY(cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        TASC_CUDA_TRY(cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 184 * 1024));
         attr = true;
     }
     ProfScope ps(K_DRAFT, static_cast<cudaStream_t>(stream));
