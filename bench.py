@@ -15,6 +15,7 @@ the results read back inside the timed region.
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import subprocess
@@ -56,19 +57,24 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """Samples SM clocks and throttle reasons with nvidia-smi (every 20 ms) from before the timed region on; the
+    samples whose time stamps fall inside the region [mark_begin, mark_end] are the ones reported."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index, self.samples, self.proc = index, [], None
+        self.t0 = self.t1 = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
+            t_wait = time.time()
+            while not self.samples and time.time() - t_wait < 3.0:      # running before the region starts
+                time.sleep(0.01)
         except OSError:
             self.proc = None
 
@@ -76,27 +82,48 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.samples.append(line.strip())
 
+    def mark_begin(self):
+        self.t0 = datetime.datetime.now()
+
+    def mark_end(self):
+        self.t1 = datetime.datetime.now()
+
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
-        sm, smax, reasons = [], None, set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = []
         for s in self.samples:
             f = [x.strip() for x in s.split(",")]
-            if len(f) < 6:
+            if len(f) < 7:
                 continue
             try:
-                sm.append(float(f[0]))
-                smax = float(f[1])
+                when = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
+            except ValueError:
+                when = None
+            try:
+                rows.append((when, float(f[1]), float(f[2]), f[3:7]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[2:6]):
+        stamped = all(r[0] is not None for r in rows) and self.t0 is not None and self.t1 is not None
+        if not stamped:                                       # time stamps in a form not understood: every sample counts
+            rows = [(self.t0, r[1], r[2], r[3]) for r in rows]
+        inside = [r for r in rows if stamped and self.t0 <= r[0] <= self.t1] if stamped else list(rows)
+        where = "inside the timed region" if stamped else "whole sampling window"
+        if not inside and rows and stamped:                   # a region shorter than the sampling period: the nearest samples
+            mid = self.t0 + (self.t1 - self.t0) / 2
+            inside = sorted(rows, key=lambda r: abs((r[0] - mid).total_seconds()))[:2]
+            where = "nearest to the timed region"
+        reasons = set()
+        for r in inside:
+            for name, val in zip(names, r[3]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        sm = [r[1] for r in inside]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": inside[0][2] if inside else None,
+                "reasons": sorted(reasons), "samples": len(sm), "sampled": where if sm else "no samples"}
 
 
 # ----------------------------------------------------------------------------------------------- replicas
@@ -327,14 +354,16 @@ def main():
     len0 = length.clone()
     launches0 = sum(b.tasc_launch_counts().values())
     sampler = ClockSampler(local_rank)
-    barrier()
     sampler.start()
+    barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark_begin()
     ev0.record()
     for _ in range(args.steps):
         run_step()
     ev1.record()
     barrier()
+    sampler.mark_end()
     clocks = sampler.stop()
     launches = (launches_per_step * args.steps) if graph is not None else sum(b.tasc_launch_counts().values()) - launches0
     b.tasc_poll_status(ws)
