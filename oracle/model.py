@@ -16,19 +16,42 @@ evaluated in float64 and rounded to the working type.
 Arithmetic is plain numpy in ``dtype`` (float32 by default, float64 for the
 pins); matrix products are numpy matmul calls, nothing is blocked or fused.
 One sequence at a time; a batch is a loop.
+
+Storage precision.  The paper fixes none; the benchmark's "decoder in bf16" configurations fix the
+storage type of the model's state: weight matrices AND the KV cache hold bf16 values (the shapes'
+``dtype`` field says so: storage type of weights and KV).  The oracle therefore receives weights that are
+already rounded to bf16 and, for a bf16 shape, rounds K (after RoPE) and V to bf16, round-to-nearest-even,
+at the moment they are written to the cache; everything is computed in ``dtype`` from those stored values.
+(With a float32 cache the logits of the 28-layer shape at a 1,024-token context move by up to 3e-2, more
+than the whole tolerance of the comparison -- the cache format is part of what is computed, not noise.)
+``kv_storage=None`` keeps the cache in ``dtype`` (float32 shapes, and the float64 pins).
 """
 from __future__ import annotations
 
 import numpy as np
 
 
-class KVCache:
-    """Per-layer K and V of one sequence: arrays [n_kv_heads, capacity, head_dim], ``length`` valid."""
+def to_bf16_storage(x):
+    """The value a bf16 memory cell holds after x is written to it: the nearest number with an 8-bit significand
+    (7 stored bits), ties to the even significand.  Computed on the float32 bit pattern: add 0x7FFF plus the lowest
+    kept bit, then clear the 16 dropped bits."""
+    bits = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    lowest_kept = (bits >> np.uint32(16)) & np.uint32(1)
+    return ((bits + np.uint32(0x7FFF) + lowest_kept) & np.uint32(0xFFFF0000)).view(np.float32)
 
-    def __init__(self, shape, capacity: int, dtype=np.float32):
+
+class KVCache:
+    """Per-layer K and V of one sequence: arrays [n_kv_heads, capacity, head_dim], ``length`` valid.
+    ``storage`` = "bf16": values are rounded to bf16 when they are written (see the module header)."""
+
+    def __init__(self, shape, capacity: int, dtype=np.float32, storage=None):
         self.k = [np.zeros((shape.n_kv_heads, capacity, shape.head_dim), dtype) for _ in range(shape.n_layers)]
         self.v = [np.zeros((shape.n_kv_heads, capacity, shape.head_dim), dtype) for _ in range(shape.n_layers)]
         self.length = 0
+        self.storage = storage
+
+    def stored(self, x):
+        return to_bf16_storage(x).astype(x.dtype) if self.storage == "bf16" else x
 
     def truncate(self, length: int):
         """Roll back: positions >= length are dead and will be overwritten."""
@@ -59,9 +82,11 @@ def silu(x):
 
 
 class OracleModel:
-    def __init__(self, shape, weights: dict, dtype=np.float32):
+    def __init__(self, shape, weights: dict, dtype=np.float32, kv_storage="shape"):
         self.s = shape
         self.dtype = dtype
+        # "shape": the cache stores what the shape's dtype says (bf16 shapes: bf16 cells); None: cells of ``dtype``
+        self.kv_storage = (("bf16" if shape.dtype == "bf16" else None) if kv_storage == "shape" else kv_storage)
         cast = lambda a: np.asarray(a, dtype=dtype)
         self.embed = cast(weights["embed"])
         self.lm_head = self.embed if weights["lm_head"] is weights["embed"] else cast(weights["lm_head"])
@@ -69,7 +94,7 @@ class OracleModel:
         self.layers = [{k: cast(v) for k, v in lw.items()} for lw in weights["layers"]]
 
     def new_cache(self, capacity: int) -> KVCache:
-        return KVCache(self.s, capacity, self.dtype)
+        return KVCache(self.s, capacity, self.dtype, self.kv_storage)
 
     def hidden(self, tokens, cache: KVCache):
         """Final-norm hidden states [R, d] of R new tokens at positions cache.length..+R-1;
@@ -90,8 +115,8 @@ class OracleModel:
             v = qkv[:, s.q_dim + s.kv_dim:].reshape(R, s.n_kv_heads, s.head_dim)
             q = apply_rope(q, cos, sin)
             k = apply_rope(k, cos, sin)
-            cache.k[l][:, p0:p0 + R] = k.transpose(1, 0, 2)
-            cache.v[l][:, p0:p0 + R] = v.transpose(1, 0, 2)
+            cache.k[l][:, p0:p0 + R] = cache.stored(k.transpose(1, 0, 2))
+            cache.v[l][:, p0:p0 + R] = cache.stored(v.transpose(1, 0, 2))
             attn = np.zeros((R, s.n_q_heads, s.head_dim), self.dtype)
             for hq in range(s.n_q_heads):
                 K = cache.k[l][hq // g, :p0 + R]

@@ -205,3 +205,49 @@ def test_bf16_rounding_is_nearest_even():
     assert np.array_equal(W.round_to_bf16(r), torch.tensor(r).to(torch.bfloat16).to(torch.float32).numpy())
     assert np.array_equal(W.bf16_bits(W.round_to_bf16(r)).view(np.int16),
                           torch.tensor(r).to(torch.bfloat16).view(torch.int16).numpy())
+
+
+def test_bf16_cache_cells_round_to_nearest_even():
+    """The oracle's own model of a bf16 memory cell against the published format: hand-picked ties and halves,
+    a library conversion (torch) on random values, and idempotence."""
+    from oracle.model import to_bf16_storage
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7 -> even (1); 1 + 3 * 2^-8 is a tie -> even (1 + 2^-6)
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -2.5, 0.0],
+                 dtype=np.float32)
+    want = np.array([1.0, 1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7, -2.5, 0.0], dtype=np.float32)
+    assert np.array_equal(to_bf16_storage(x), want)
+    r = (np.random.default_rng(1).standard_normal(20000) * np.float32(37.0)).astype(np.float32)
+    got = to_bf16_storage(r)
+    assert np.array_equal(got, torch.tensor(r).to(torch.bfloat16).to(torch.float32).numpy())
+    assert np.array_equal(to_bf16_storage(got), got)
+    assert np.all(np.abs(got - r) <= np.abs(r) * 2.0 ** -8)            # half a unit in the last of 8 significand bits
+
+
+def test_bf16_shapes_store_their_cache_in_bf16_and_float32_shapes_do_not():
+    from dataclasses import replace
+    from oracle.model import to_bf16_storage
+    shape16 = replace(SHAPE, dtype="bf16")
+    w = W.make_weights(shape16, seed=3, gain_jitter=0.2)
+    toks = [3, 14, 15, 9, 2, 6]
+    m16 = OracleModel(shape16, w, np.float32)
+    c16 = m16.new_cache(8)
+    m16.forward(toks, c16)
+    for l in range(shape16.n_layers):                                   # every cell holds a bf16 value
+        assert np.array_equal(to_bf16_storage(c16.k[l]), c16.k[l]) and np.array_equal(to_bf16_storage(c16.v[l]), c16.v[l])
+    # what is stored is the rounding of what the float32-cache model computes for the first layer ...
+    m32 = OracleModel(shape16, w, np.float32, kv_storage=None)
+    c32 = m32.new_cache(8)
+    m32.forward(toks, c32)
+    assert np.array_equal(c16.k[0], to_bf16_storage(c32.k[0])) and np.array_equal(c16.v[0], to_bf16_storage(c32.v[0]))
+    assert not np.array_equal(c32.k[0], c16.k[0])
+    # ... incremental decoding reads the same stored cells as the one-pass forward: identical logits up to the
+    # float32 order of operations, and a rolled-back cache recomputes the same cells
+    c_inc = m16.new_cache(8)
+    inc = np.concatenate([m16.forward([t], c_inc) for t in toks])
+    c_one = m16.new_cache(8)
+    one = m16.forward(toks, c_one)
+    assert np.abs(inc - one).max() < 1e-5
+    assert all(np.array_equal(c_inc.k[l][:, :6], c_one.k[l][:, :6]) for l in range(shape16.n_layers))
+    # a float32 shape keeps float32 cells
+    c = OracleModel(SHAPE, w, np.float32).new_cache(8)
+    assert c.storage is None
