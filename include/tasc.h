@@ -40,6 +40,7 @@ typedef int32_t tasc_status;
 #define TASC_MAX_ORDER   5    /* largest context length n_max of the n-gram models */
 #define TASC_MAX_ROWS   16    /* largest k + 1 (rows verified per sequence per step) */
 #define TASC_VOCAB_BITS 20    /* token ids must be < 2^20 (six ids + order are packed in 128 bits) */
+#define TASC_TOK_MAX_N    6    /* longest n-gram the tokenizer enrichment merges into one token */
 
 #define TASC_F32   0
 #define TASC_BF16  1
@@ -69,6 +70,9 @@ typedef struct {
  *   n_max          1..TASC_MAX_ORDER;  p_min >= 1 (absolute count threshold)
  *   vocab          <= 2^TASC_VOCAB_BITS
  *   out            host; receives a handle owning device tables (tasc_drafter_destroy)
+ * Device memory: the tables the handle owns (about 40 bytes per surviving element), and, while the call runs,
+ * a counting table of 2^ceil(log2(2 W)) slots of 20 bytes, W = the windows of order 1 (tokens minus documents), plus
+ * one byte per token -- about 5.4 GB for a corpus of 110 M tokens; freed before the call returns.
  * Synchronises the stream before returning.  Errors: EINVAL, ENOMEM, ECUDA,
  * ECAPACITY (internal table overflow; not expected for valid input).
  */
@@ -101,11 +105,109 @@ tasc_status tasc_drafter_destroy(tasc_drafter* d);
  *   drafts   device, int32[B][k] (written)
  *   k        1..TASC_MAX_ROWS-1;  0 <= lambda_num <= lambda_den <= 256
  * Asynchronous on the stream.  Errors: EINVAL (also when stride is too large for the
- * kernel's shared-memory successor table: stride <= 12288).
+ * kernel's shared-memory copy of the tokens and successor table: stride <= 12288, which is therefore the
+ * longest context -- prompt plus generated tokens plus k + 1 -- the whole path supports).
  */
 tasc_status tasc_draft(const tasc_drafter* d, const int32_t* tokens, int64_t stride, const int32_t* len,
                        int32_t B, int32_t k, int32_t lambda_num, int32_t lambda_den, int32_t* drafts,
                        tasc_stream stream);
+
+/*
+ * The comparison drafter of Section 6.2 (the "N-Grammys" bigram: for every token of the vocabulary the most probable
+ * next token under the target model's own conditional distribution) as a drafter handle: an order-1 model in which
+ * context token c has the single successor table[c] with count 1.  tasc_draft then mixes it with the context drafter
+ * exactly as it mixes p_corp (a point mass in the place of p_corp: for lambda >= 1/2 it always wins; with a small
+ * lambda the context drafter decides wherever it has a match and the bigram elsewhere).  The last-resort token is 0.
+ *
+ *   table   device, int32[vocab], every entry in [0, vocab) (tasc_bigram_table writes one)
+ *   out     host; receives a handle owning device tables (tasc_drafter_destroy)
+ * Synchronises the stream.  Errors: EINVAL (also for an entry outside the vocabulary), ENOMEM, ECUDA.
+ */
+tasc_status tasc_drafter_from_bigram(const int32_t* table, int32_t vocab, tasc_stream stream, tasc_drafter** out);
+
+/*
+ * Statistics of the task's output corpus C_task (Section 3: the concentration of the task-conditioned n-gram
+ * distribution, Eq. 1-2, reported in Table 1 as the bigram Shannon entropy and the number of distinct bigrams
+ * that cover 80 % of the bigram occurrences; Section 4.1 / Appendix "Uniform Information Density": the token
+ * entropy divided by log |V|; Section 6.1 / Appendix "Predicting Model Speedup": the Renyi entropy of order 2 of
+ * the token distribution, H_2 = -log sum_x p(x)^2).  A bigram is an adjacent token pair inside one document --
+ * the windows of the order-1 model before pruning.  Entropies are in bits; typical_set_size = 2^H (Eq. 2).
+ */
+typedef struct {
+    int64_t n_tokens;                 /* tokens of the corpus */
+    int64_t n_bigrams;                /* bigram occurrences: sum over documents of max(0, length - 1) */
+    int64_t n_unique_tokens;
+    int64_t n_unique_bigrams;
+    int64_t bigrams_for_cdf;          /* smallest m: the m most frequent bigrams hold >= cdf_num / cdf_den of n_bigrams */
+    double  bigram_entropy_bits;
+    double  typical_set_size;
+    double  token_entropy_bits;
+    double  token_entropy_normalised; /* token_entropy_bits / log2(vocab) */
+    double  token_renyi2_bits;
+} tasc_corpus_statistics;
+
+/*
+ *   corpus_tokens, doc_offsets, n_docs, vocab   as for tasc_drafter_build (device pointers)
+ *   cdf_num / cdf_den   coverage target of bigrams_for_cdf (the paper's 80 % = 4 / 5); 1 <= cdf_num <= cdf_den <= 65536
+ *   out                 host (written)
+ * Counting and the reductions run on the device; the integer fields are exact and, like the entropies, do not depend
+ * on thread timing.  Allocates transient device memory (about 40 bytes per bigram occurrence plus 8 MiB) and frees it
+ * before returning; synchronises the stream.  The corpus must hold fewer than 2^40 tokens.
+ * Errors: EINVAL, ENOMEM, ECUDA, ECAPACITY (more than 4,096 distinct bigrams or tokens occurring 2^20 times or more).
+ */
+tasc_status tasc_corpus_stats(const int32_t* corpus_tokens, const int64_t* doc_offsets, int64_t n_docs, int32_t vocab,
+                              int32_t cdf_num, int32_t cdf_den, tasc_stream stream, tasc_corpus_statistics* out);
+
+/* ------------------------------------------------------- tokenizer enrichment */
+
+/*
+ * Algorithm 1 of the paper (Section 4.1, "Tokenizer Enrichment"): starting from the base vocabulary, repeat `budget`
+ * times: collect the token n-grams (2 <= n <= n_max) of the task corpus as tokenised with the current vocabulary,
+ * score each with the merge reward f_merge(t^n) = freq(t^n) * (n - 1), add the argmax as one new token (id
+ * base_vocab + i for the i-th addition) and replace its occurrences -- left to right, non-overlapping, inside each
+ * document -- before the next round.  freq counts every window; windows do not span documents; argmax ties go to the
+ * longer n-gram, then to the one that occurs first.  The prefix-collision test needs token strings and is not applied.
+ * Stops early when no n-gram is left.
+ *
+ *   corpus_tokens, doc_offsets, n_docs   as for tasc_drafter_build (device); ids in [0, base_vocab); fewer than 2^28 tokens
+ *   budget        additions M (base_vocab + budget <= 2^TASC_VOCAB_BITS);  n_max  2..TASC_TOK_MAX_N
+ *   merges        device, int32[budget][TASC_TOK_MAX_N] (written): the constituents of each added token, ids of the
+ *                 vocabulary at the time of the merge (a constituent may be an earlier added token), padded with -1
+ *   n_merges      host (written): additions made
+ *   tokens_out    device, int32[doc_offsets[n_docs]] (written): the corpus in the enriched vocabulary, compacted
+ *   offsets_out   device, int64[n_docs + 1] (written)
+ * Every round recounts the whole corpus: the cost is budget x corpus size, so select on a sample of the corpus.
+ * Allocates transient device memory (about 50 bytes per n-gram window) and frees it; synchronises the stream.
+ * Errors: EINVAL, ENOMEM, ECUDA, ECAPACITY.
+ */
+tasc_status tasc_tok_enrich(const int32_t* corpus_tokens, const int64_t* doc_offsets, int64_t n_docs, int32_t base_vocab,
+                            int32_t budget, int32_t n_max, int32_t* merges, int32_t* n_merges, int32_t* tokens_out,
+                            int64_t* offsets_out, tasc_stream stream);
+
+/*
+ * Rows of the added tokens for the embedding or the LM-head matrix (Section 4.2): e_new = (1/n) sum_j e_{t_j} over the n
+ * constituents, summed in float32 in their order and divided by n, stored in the matrix's type (bf16: nearest even).
+ *   matrix   device, [base_vocab][d] in `dtype` (TASC_F32 / TASC_BF16);  merges as written by tasc_tok_enrich
+ *   rows_out device, [n_merges][d] in `dtype` (written; also read, for constituents that are added tokens)
+ *   device_status  device, int32, zeroed by the caller: TASC_EINVAL if a merge names a token that does not exist yet
+ * Asynchronous.  Errors: EINVAL.
+ */
+tasc_status tasc_tok_init_rows(const void* matrix, int32_t dtype, int32_t base_vocab, int32_t d, const int32_t* merges,
+                               int32_t n_merges, void* rows_out, int32_t* device_status, tasc_stream stream);
+
+/*
+ * Encode base-token text with the enriched vocabulary (the paper's appendix on byte-pair encoding: the added tokens are
+ * queried before the base tokenizer): at every position the added token with the longest expansion into base tokens
+ * that matches the upcoming tokens (and ends inside the document) replaces them; elsewhere the base token stays.
+ * Two added tokens with the same expansion: the earlier one.
+ *   tokens, doc_offsets, n_docs   device, base-vocabulary text;  merges, n_merges as above (device)
+ *   tokens_out   device, room for as many tokens as the input (written, compacted);  offsets_out device, int64[n_docs + 1]
+ * The trie of the expansions is built on the host from the merge list (expansions of more than 4,096 base tokens:
+ * ECAPACITY).  Allocates transient device memory; synchronises the stream.  Errors: EINVAL, ENOMEM, ECUDA, ECAPACITY.
+ */
+tasc_status tasc_tok_encode(const int32_t* tokens, const int64_t* doc_offsets, int64_t n_docs, int32_t base_vocab,
+                            const int32_t* merges, int32_t n_merges, int32_t* tokens_out, int64_t* offsets_out,
+                            tasc_stream stream);
 
 /* -------------------------------------------------------------------- model */
 
@@ -234,6 +336,22 @@ tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* d, const tasc
                           int32_t B, int32_t max_new, const tasc_draft_params* params, int32_t* out,
                           tasc_stats* stats, void* workspace, size_t workspace_bytes, tasc_stream stream);
 
+/*
+ * The bigram table of the comparison drafter of Section 6.2 ("N-Grammys": a bigram model obtained by taking the target
+ * model's conditional distribution for each element of the vocabulary): table[t] = argmax over x of the model's logits
+ * for the single-token context t (position 0, no earlier keys), smallest id on ties.  The vocabulary runs through the
+ * verify forward (every layer, LM head, row argmax) as passes of B one-row sequences.
+ *
+ *   kv         a pool in which each of the B sequences has at least one page (block_table as for tasc_verify_step);
+ *              its contents are overwritten
+ *   B          single-token sequences per pass (1 .. as many as workspace and kv were sized for)
+ *   table      device, int32[vocab] (written)
+ *   workspace  at least tasc_workspace_bytes(m, B, 1) bytes
+ * Asynchronous (ceil(vocab / B) forward passes are enqueued).  Errors: EINVAL; device-side statuses via tasc_poll_status.
+ */
+tasc_status tasc_bigram_table(const tasc_model* m, const tasc_kv* kv, int32_t B, int32_t* table, void* workspace,
+                              size_t workspace_bytes, tasc_stream stream);
+
 /* Synchronise the stream and return the device status word of the workspace (TASC_OK if clean); clears it. */
 tasc_status tasc_poll_status(void* workspace, tasc_stream stream);
 
@@ -282,7 +400,10 @@ size_t tasc_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
  *
  *   x, w, y, M, N, K   as tasc_gemm_bf16
  *   device_status      device, int32, or NULL: receives a device-side error code of this call (0 = none),
- *                      cleared at the start of the call; with NULL the word lives inside the shared array
+ *                      cleared at the start of the call.  With NULL the word lives inside the shared array
+ *                      where no call can read it back: a device-side error (a bounded wait that ran out,
+ *                      TASC_ETIMEOUT) then goes unreported and y holds zeros for the affected tiles -- pass
+ *                      a status word if the result must be trusted.
  * Limits and rules:
  *   - the float32 partial sums (k-splits * M * N * 4 bytes) must fit in 8 MiB minus 256 bytes; the call takes
  *     fewer k-splits than tasc_gemm_bf16 if that makes them fit (only the summation order changes) and

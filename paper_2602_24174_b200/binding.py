@@ -24,7 +24,7 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ENOKV, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
-MAX_ORDER, MAX_ROWS, VOCAB_BITS = 5, 16, 20
+MAX_ORDER, MAX_ROWS, VOCAB_BITS, TOK_MAX_N = 5, 16, 20, 6
 F32, BF16 = 0, 1
 MODE_GREEDY, MODE_CONTINUATION, MODE_FORCED_ACCEPT = 0, 1, 2
 
@@ -60,6 +60,12 @@ class Seqs(C.Structure):
     _fields_ = [("tokens", C.c_void_p), ("stride", C.c_int64), ("len", C.c_void_p), ("stop_len", C.c_void_p)]
 
 
+class CorpusStatistics(C.Structure):
+    _fields_ = [("n_tokens", C.c_int64), ("n_bigrams", C.c_int64), ("n_unique_tokens", C.c_int64), ("n_unique_bigrams", C.c_int64),
+                ("bigrams_for_cdf", C.c_int64), ("bigram_entropy_bits", C.c_double), ("typical_set_size", C.c_double),
+                ("token_entropy_bits", C.c_double), ("token_entropy_normalised", C.c_double), ("token_renyi2_bits", C.c_double)]
+
+
 class DraftParams(C.Structure):
     _fields_ = [("k", C.c_int32), ("lambda_num", C.c_int32), ("lambda_den", C.c_int32), ("mode", C.c_int32),
                 ("forced_accept", C.c_int32), ("continuation", C.c_void_p), ("continuation_stride", C.c_int64)]
@@ -77,6 +83,18 @@ lib.tasc_last_error.restype = C.c_char_p
 lib.tasc_drafter_build.argtypes = [_P, _P, C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(_P)]
 lib.tasc_drafter_export.argtypes = [_P, C.POINTER(NgramEntry), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 lib.tasc_drafter_destroy.argtypes = [_P]
+lib.tasc_drafter_from_bigram.argtypes = [_P, C.c_int32, _P, C.POINTER(_P)]
+lib.tasc_drafter_from_bigram.restype = C.c_int32
+lib.tasc_bigram_table.argtypes = [_P, C.POINTER(Kv), C.c_int32, _P, _P, C.c_size_t, _P]
+lib.tasc_bigram_table.restype = C.c_int32
+lib.tasc_tok_enrich.argtypes = [_P, _P, C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(C.c_int32), _P, _P, _P]
+lib.tasc_tok_enrich.restype = C.c_int32
+lib.tasc_tok_init_rows.argtypes = [_P, C.c_int32, C.c_int32, C.c_int32, _P, C.c_int32, _P, _P, _P]
+lib.tasc_tok_init_rows.restype = C.c_int32
+lib.tasc_tok_encode.argtypes = [_P, _P, C.c_int64, C.c_int32, _P, C.c_int32, _P, _P, _P]
+lib.tasc_tok_encode.restype = C.c_int32
+lib.tasc_corpus_stats.argtypes = [_P, _P, C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(CorpusStatistics)]
+lib.tasc_corpus_stats.restype = C.c_int32
 lib.tasc_draft.argtypes = [_P, _P, C.c_int64, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P, _P]
 lib.tasc_model_create.argtypes = [C.POINTER(ModelDesc), C.POINTER(Weights), C.POINTER(_P)]
 lib.tasc_model_destroy.argtypes = [_P]
@@ -164,6 +182,78 @@ def tasc_drafter_build(corpus_tokens: torch.Tensor, doc_offsets: torch.Tensor, n
     return Drafter(h, n_max)
 
 
+def tasc_drafter_from_bigram(table: torch.Tensor, vocab: int) -> Drafter:
+    """Drafter handle of the model-derived bigram (context token c -> table[c])."""
+    _dev(table, torch.int32)
+    assert table.numel() == vocab
+    h = _P()
+    _check(lib.tasc_drafter_from_bigram(_ptr(table), vocab, _stream(), C.byref(h)), "tasc_drafter_from_bigram")
+    return Drafter(h, 1)
+
+
+def tasc_bigram_table(model: "Model", kv: "Kv", B: int, workspace: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """table[t] = the model's most probable next token after the single-token context t (int32[vocab] CUDA tensor)."""
+    if out is None:
+        out = torch.empty(model.shape.vocab, dtype=torch.int32, device=workspace.device)
+    _dev(out, torch.int32)
+    _check(lib.tasc_bigram_table(model._h, C.byref(kv), B, _ptr(out), _ptr(workspace), workspace.numel(), _stream()),
+           "tasc_bigram_table")
+    return out
+
+
+def tasc_tok_enrich(corpus_tokens: torch.Tensor, doc_offsets: torch.Tensor, base_vocab: int, budget: int, n_max: int):
+    """Algorithm 1.  Returns (merges int32[n_merges, TOK_MAX_N] padded with -1, tokens, offsets) as CUDA tensors."""
+    _dev(corpus_tokens, torch.int32)
+    _dev(doc_offsets, torch.int64)
+    dev = doc_offsets.device
+    merges = torch.empty((max(budget, 1), TOK_MAX_N), dtype=torch.int32, device=dev)
+    toks = torch.empty(max(corpus_tokens.numel(), 1), dtype=torch.int32, device=dev)
+    offs = torch.empty(doc_offsets.numel(), dtype=torch.int64, device=dev)
+    n = C.c_int32(0)
+    _check(lib.tasc_tok_enrich(_ptr(corpus_tokens), _ptr(doc_offsets), doc_offsets.numel() - 1, base_vocab, budget, n_max,
+                               _ptr(merges), C.byref(n), _ptr(toks), _ptr(offs), _stream()), "tasc_tok_enrich")
+    total = int(offs[-1].item())
+    return merges[:n.value], toks[:total], offs
+
+
+def tasc_tok_init_rows(matrix: torch.Tensor, merges: torch.Tensor) -> torch.Tensor:
+    """Rows of the added tokens (mean of the constituents' rows) for an embedding / LM-head matrix [base_vocab, d]."""
+    assert matrix.is_cuda and matrix.is_contiguous() and matrix.dtype in (torch.float32, torch.bfloat16)
+    _dev(merges, torch.int32)
+    base_vocab, d = matrix.shape
+    rows = torch.zeros((merges.shape[0], d), dtype=matrix.dtype, device=matrix.device)
+    status = torch.zeros(1, dtype=torch.int32, device=matrix.device)
+    _check(lib.tasc_tok_init_rows(_ptr(matrix), F32 if matrix.dtype == torch.float32 else BF16, base_vocab, d, _ptr(merges),
+                                  merges.shape[0], _ptr(rows), _ptr(status), _stream()), "tasc_tok_init_rows")
+    code = int(status.item())
+    if code != OK:
+        raise TascError(code, "tasc_tok_init_rows (device)")
+    return rows
+
+
+def tasc_tok_encode(tokens: torch.Tensor, doc_offsets: torch.Tensor, base_vocab: int, merges: torch.Tensor):
+    """Greedy longest-match encoding with the added tokens first.  Returns (tokens, offsets)."""
+    _dev(tokens, torch.int32)
+    _dev(doc_offsets, torch.int64)
+    _dev(merges, torch.int32)
+    dev = doc_offsets.device
+    toks = torch.empty(max(tokens.numel(), 1), dtype=torch.int32, device=dev)
+    offs = torch.empty(doc_offsets.numel(), dtype=torch.int64, device=dev)
+    _check(lib.tasc_tok_encode(_ptr(tokens), _ptr(doc_offsets), doc_offsets.numel() - 1, base_vocab, _ptr(merges), merges.shape[0],
+                               _ptr(toks), _ptr(offs), _stream()), "tasc_tok_encode")
+    return toks[:int(offs[-1].item())], offs
+
+
+def tasc_corpus_stats(corpus_tokens: torch.Tensor, doc_offsets: torch.Tensor, vocab: int, cdf_num: int = 4, cdf_den: int = 5) -> dict:
+    """Corpus statistics as a dict with the field names of tasc_corpus_statistics."""
+    _dev(corpus_tokens, torch.int32)
+    _dev(doc_offsets, torch.int64)
+    out = CorpusStatistics()
+    _check(lib.tasc_corpus_stats(_ptr(corpus_tokens), _ptr(doc_offsets), doc_offsets.numel() - 1, vocab, cdf_num, cdf_den,
+                                 _stream(), C.byref(out)), "tasc_corpus_stats")
+    return {name: getattr(out, name) for name, _ in CorpusStatistics._fields_}
+
+
 def tasc_draft(drafter: Drafter, tokens: torch.Tensor, length: torch.Tensor, k: int, lambda_num: int = 3,
                lambda_den: int = 4, out: torch.Tensor | None = None) -> torch.Tensor:
     _dev(tokens, torch.int32)
@@ -247,15 +337,26 @@ def tasc_prefill(model: Model, kv: Kv, seqs: Seqs, B: int, max_len: int, workspa
 
 
 def tasc_verify_step(model: Model, kv: Kv, seqs: Seqs, drafts: torch.Tensor, workspace: torch.Tensor, *,
-                     forced_targets: torch.Tensor | None = None, want_targets: bool = False, want_logits: bool = False):
-    """Returns (n_accepted[B], next_token[B], target_tokens[B, k+1] or None, logits[B, k+1, V] or None)."""
+                     forced_targets: torch.Tensor | None = None, want_targets: bool = False, want_logits: bool = False,
+                     out: tuple | None = None):
+    """Returns (n_accepted[B], next_token[B], target_tokens[B, k+1] or None, logits[B, k+1, V] or None).
+    ``out``: caller-provided (n_accepted, next_token, target_tokens or None, logits or None) to write into."""
     _dev(drafts, torch.int32)
     B, k = drafts.shape
     dev = drafts.device
-    n_acc = torch.empty(B, dtype=torch.int32, device=dev)
-    nxt = torch.empty(B, dtype=torch.int32, device=dev)
-    tgt = torch.empty((B, k + 1), dtype=torch.int32, device=dev) if want_targets else None
-    logits = torch.empty((B, k + 1, model.shape.vocab), dtype=torch.float32, device=dev) if want_logits else None
+    if out is not None:
+        n_acc, nxt, tgt, logits = out
+        assert tuple(n_acc.shape) == (B,) and tuple(nxt.shape) == (B,)
+        assert tgt is None or tuple(tgt.shape) == (B, k + 1)
+        assert logits is None or tuple(logits.shape) == (B, k + 1, model.shape.vocab)
+        for t, dt in ((n_acc, torch.int32), (nxt, torch.int32), (tgt, torch.int32), (logits, torch.float32)):
+            if t is not None:
+                _dev(t, dt)
+    else:
+        n_acc = torch.empty(B, dtype=torch.int32, device=dev)
+        nxt = torch.empty(B, dtype=torch.int32, device=dev)
+        tgt = torch.empty((B, k + 1), dtype=torch.int32, device=dev) if want_targets else None
+        logits = torch.empty((B, k + 1, model.shape.vocab), dtype=torch.float32, device=dev) if want_logits else None
     if forced_targets is not None:
         _dev(forced_targets, torch.int32)
     _check(lib.tasc_verify_step(model._h, C.byref(kv), C.byref(seqs), _ptr(drafts), B, k, _ptr(forced_targets), _ptr(n_acc),

@@ -4,8 +4,21 @@
 #include "kernels.h"
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
+
+// Launch shapes and activation tensor maps of one forward of a bf16 model, which depend only on the row counts, the
+// cache capacity and the workspace address: planned once and reused by every later step on the same buffers.
+struct StepPlans {
+    int B, R, max_ctx;
+    const void* ws_h;
+    tasc::AttnPlan att;
+    int TB;
+    uint64_t rows;
+    CUtensorMap tm_h, tm_o, tm_act, tm_h_lm;
+    tasc::FusedPlan p_qkv, p_o, p_gu, p_down, p_lm;
+};
 
 struct tasc_model {
     tasc_model_desc desc;
@@ -19,6 +32,9 @@ struct tasc_model {
     std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
     CUtensorMap tm_lm;
     int qkv_rows, q_dim, kv_dim;
+    int few_tiles;                                  // token tiles for 49..128 rows (see gemm_token_tile), from the layer's weight bytes
+    mutable std::mutex plan_mu;
+    mutable std::vector<StepPlans> plans;           // most recently used last; a handful of (B, k, workspace) combinations
 };
 
 namespace tasc {
@@ -187,21 +203,39 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
     const tasc_model_desc& d = m->desc;
     const int M = B * R;
     const int max_ctx = kv->max_pages_per_seq * d.page_size;
-    // attention works on blocks of at most 16 rows per sequence (one block in a verify step, several in a prefill pass)
-    const int att_rows = R <= 16 ? R : 16;
-    const AttnPlan att_plan = plan_attention_mma(B * (R / att_rows), d.n_kv_heads, d.head_dim,
-                                                 (d.n_q_heads / d.n_kv_heads) * att_rows, max_ctx);
-    const int TB = gemm_token_tile(M, true);
-    const uint64_t rows = (uint64_t)((M + TB - 1) / TB) * 2 * TB;
-    CUtensorMap tm_h, tm_o, tm_act;
     tasc_status st;
-    if ((st = encode_tmap_bf16(&tm_h, w.h, rows, d.d_model, 2 * TB)) != TASC_OK) return st;
-    if ((st = encode_tmap_bf16(&tm_o, w.o, rows, m->q_dim, 2 * TB)) != TASC_OK) return st;
-    if ((st = encode_tmap_bf16(&tm_act, w.act, rows, d.d_ff, 2 * TB)) != TASC_OK) return st;
-    const FusedPlan p_qkv = plan_fused(M, m->qkv_rows, d.d_model, EPI_QKV);
-    const FusedPlan p_o = plan_fused(M, d.d_model, m->q_dim, EPI_RESID);
-    const FusedPlan p_gu = plan_fused(M, d.d_ff, d.d_model, EPI_SWIGLU);
-    const FusedPlan p_down = plan_fused(M, d.d_model, d.d_ff, EPI_RESID);
+    StepPlans sp;
+    {
+        std::lock_guard<std::mutex> lk(m->plan_mu);
+        auto it = std::find_if(m->plans.begin(), m->plans.end(), [&](const StepPlans& c) {
+            return c.B == B && c.R == R && c.max_ctx == max_ctx && c.ws_h == w.h; });
+        if (it != m->plans.end()) {
+            sp = *it;
+        } else {
+            sp.B = B; sp.R = R; sp.max_ctx = max_ctx; sp.ws_h = w.h;
+            // attention works on blocks of at most 16 rows per sequence (one block in a verify step, several in a prefill pass)
+            const int att_rows = R <= 16 ? R : 16;
+            sp.att = plan_attention_mma(B * (R / att_rows), d.n_kv_heads, d.head_dim, d.n_q_heads / d.n_kv_heads, att_rows, max_ctx);
+            sp.TB = gemm_token_tile(M, true, m->few_tiles);
+            sp.rows = (uint64_t)((M + sp.TB - 1) / sp.TB) * 2 * sp.TB;
+            if ((st = encode_tmap_bf16(&sp.tm_h, w.h, sp.rows, d.d_model, 2 * sp.TB)) != TASC_OK) return st;
+            if ((st = encode_tmap_bf16(&sp.tm_o, w.o, sp.rows, m->q_dim, 2 * sp.TB)) != TASC_OK) return st;
+            if ((st = encode_tmap_bf16(&sp.tm_act, w.act, sp.rows, d.d_ff, 2 * sp.TB)) != TASC_OK) return st;
+            sp.p_qkv = plan_fused(M, m->qkv_rows, d.d_model, EPI_QKV, m->few_tiles);
+            sp.p_o = plan_fused(M, d.d_model, m->q_dim, EPI_RESID, m->few_tiles);
+            sp.p_gu = plan_fused(M, d.d_ff, d.d_model, EPI_SWIGLU, m->few_tiles);
+            sp.p_down = plan_fused(M, d.d_model, d.d_ff, EPI_RESID, m->few_tiles);
+            sp.p_lm = plan_fused(M, d.vocab, d.d_model, EPI_LM, m->few_tiles);
+            // the LM head's CTAs take several layout tiles at once
+            if ((st = encode_tmap_bf16(&sp.tm_h_lm, w.h, sp.rows, d.d_model, sp.p_lm.BN)) != TASC_OK) return st;
+            if (m->plans.size() >= 16) m->plans.erase(m->plans.begin());
+            m->plans.push_back(sp);
+        }
+    }
+    const AttnPlan& att_plan = sp.att;
+    const int TB = sp.TB;
+    const CUtensorMap &tm_h = sp.tm_h, &tm_o = sp.tm_o, &tm_act = sp.tm_act;
+    const FusedPlan &p_qkv = sp.p_qkv, &p_o = sp.p_o, &p_gu = sp.p_gu, &p_down = sp.p_down;
     __nv_bfloat16* h = static_cast<__nv_bfloat16*>(w.h);
     __nv_bfloat16* o = static_cast<__nv_bfloat16*>(w.o);
     __nv_bfloat16* act = static_cast<__nv_bfloat16*>(w.act);
@@ -248,9 +282,8 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
         if ((st = launch_gemm_fused(EPI_RESID, &m->tm_down[l], &tm_act, a, p_down, s)) != TASC_OK) return st;
     }
     if (lm_head) {
-        const FusedPlan p_lm = plan_fused(M, d.vocab, d.d_model, EPI_LM);
-        CUtensorMap tm_h_lm;                       // the LM head's CTAs take several layout tiles at once
-        if ((st = encode_tmap_bf16(&tm_h_lm, w.h, rows, d.d_model, p_lm.BN)) != TASC_OK) return st;
+        const FusedPlan& p_lm = sp.p_lm;
+        const CUtensorMap& tm_h_lm = sp.tm_h_lm;
         FusedArgs a = base;
         a.N = d.vocab; a.K = d.d_model; a.ssq_in = w.ssq; a.argmax = w.argmax; a.logits = logits;
         if ((st = launch_gemm_fused(EPI_LM, &m->tm_lm, &tm_h_lm, a, p_lm, s)) != TASC_OK) return st;
@@ -326,6 +359,12 @@ extern "C" tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc
     m->q_dim = d.n_q_heads * d.head_dim;
     m->kv_dim = d.n_kv_heads * d.head_dim;
     m->qkv_rows = m->q_dim + 2 * m->kv_dim;
+    {
+        // every extra token tile streams the layer's weights once more (about 0.15 us per MB) and saves about 7 us of
+        // exchange and epilogue time per layer: below 24 MB three tiles, below 60 MB two, above that one
+        const double layer_mb = 2.0 * ((double)m->qkv_rows * d.d_model + (double)d.d_model * m->q_dim + 3.0 * d.d_ff * d.d_model) / 1e6;
+        m->few_tiles = layer_mb < 24.0 ? 3 : (layer_mb < 60.0 ? 2 : 1);
+    }
     m->rope = nullptr;
     for (int l = 0; l < d.n_layers; ++l) {
         if (!wt->attn_norm[l] || !wt->wqkv[l] || !wt->wo[l] || !wt->mlp_norm[l] || !wt->w_gate_up[l] || !wt->w_down[l]) {
@@ -498,6 +537,27 @@ extern "C" tasc_status tasc_generate(const tasc_model* m, const tasc_drafter* dr
     return st;
 }
 
+extern "C" tasc_status tasc_bigram_table(const tasc_model* m, const tasc_kv* kv, int32_t B, int32_t* table, void* workspace,
+                                         size_t workspace_bytes, tasc_stream stream) {
+    if (!m || !kv || !table || !workspace || B < 1) return TASC_EINVAL;
+    if (!kv->pool || !kv->block_table || kv->n_pages < 1 || kv->max_pages_per_seq < 1) return TASC_EINVAL;
+    if (reinterpret_cast<uintptr_t>(workspace) % ALIGN || workspace_bytes < layout_workspace(m, B, workspace).bytes) return TASC_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const Workspace w = layout_workspace(m, B, workspace);
+    const int V = m->desc.vocab;
+    // B single-token sequences per pass: each row is the whole context of its sequence (position 0, its own key only)
+    tasc_seqs seqs;
+    seqs.tokens = w.targets; seqs.stride = 1; seqs.len = w.n_accepted; seqs.stop_len = nullptr;
+    for (int t0 = 0; t0 < V; t0 += B) {
+        launch_bigram_rows(w.targets, w.n_accepted, t0, V, B, s);
+        tasc_status st = forward_any(m, kv, w, RowSource{&seqs, nullptr, -1}, B, 1, true, nullptr, s);
+        if (st != TASC_OK) return st;
+        launch_bigram_store(w.argmax, table, t0, V, B, s);
+    }
+    TASC_CUDA_TRY(cudaGetLastError());
+    return TASC_OK;
+}
+
 extern "C" tasc_status tasc_poll_status(void* workspace, tasc_stream stream) {
     if (!workspace) return TASC_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -537,6 +597,7 @@ extern "C" tasc_status tasc_gemm_bf16(const void* x, const void* wt, float* y, i
     if ((st = encode_tmap_bf16(&tmW, wt, N, K, 128)) != TASC_OK) return st;
     if ((st = encode_tmap_bf16(&tmX, x, M, K, p.BN)) != TASC_OK) return st;
     int* status = static_cast<int*>(workspace);
+    TASC_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));          // a reused workspace must not report an old error
     float* partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + 256);
     if ((st = launch_gemm_bf16(&tmW, &tmX, partials, M, N, K, p, status, s)) != TASC_OK) return st;
     launch_sum_partials(partials, p.splits, y, (size_t)M * N, s);
@@ -553,6 +614,7 @@ extern "C" tasc_status tasc_gemm_bf16x2(const float* x, const void* wt, float* y
     // the forward's kernel with the plain epilogue: split-K inside a cluster, no partial sums in global memory
     const FusedPlan p = plan_fused(M, N, K, EPI_PLAIN);
     int* status = static_cast<int*>(workspace);
+    TASC_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + 256);
     const uint64_t rows = (uint64_t)p.m_tiles * p.BN;
     TASC_CUDA_TRY(cudaMemsetAsync(xs, 0, rows * K * 2, s));

@@ -44,6 +44,7 @@ struct AttnArgs {
     int TB;
     int R, n_q, n_kv, splits, stages;  // R: rows per sequence in this pass
     int Rs, n_sub;                     // a CTA takes Rs of them (sub-block blockIdx.z % n_sub); R = Rs * n_sub
+    int hs, n_hsplit;                  // a CTA takes hs of the g query heads of its KV head (blockIdx.y % n_hsplit); g = hs * n_hsplit
     int use_tma;                       // K/V tiles by TMA box loads (16-token pages); otherwise by cp.async
     int* status;
     float scale_log2e;
@@ -94,11 +95,13 @@ __device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32
 // bandwidth; a shallower ring lets two CTAs share an SM when many (sequence, KV head) pairs are in flight.
 template <int HD, int NS> struct Ring { static constexpr int MAX_STAGES = HD >= 128 ? (NS > 4 ? 4 : 5) : 8; };
 
-// Warp groups of an eight-warp CTA whose query tile has n_slabs slabs (each group needs two ring stages).
-__host__ __device__ inline int warp_groups(int n_slabs, int stages) {
+// Warp groups of an eight-warp CTA whose query tile has n_slabs slabs and whose key range has n_tiles tiles: as many
+// groups as the warps allow, provided that each keeps two ring stages (one computing, one in flight) -- or that the
+// whole range fits the ring at once, in which case nothing is streamed behind the computation anyway.
+__host__ __device__ inline int warp_groups(int n_slabs, int stages, int n_tiles) {
     int ng = 8 / n_slabs;
     ng = ng >= 4 ? 4 : (ng >= 2 ? 2 : 1);
-    while (ng > 1 && stages / ng < 2) ng >>= 1;
+    while (ng > 1 && stages / ng < 2 && !(stages / ng >= 1 && n_tiles <= (stages / ng) * ng)) ng >>= 1;
     return ng;
 }
 
@@ -135,12 +138,13 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     __shared__ int s_pages[MAX_STAGED_PAGES];
     __shared__ uint64_t s_full[8];               // one per ring stage: bytes of its K and V tile have landed (TMA path)
 
-    const int sp = blockIdx.x, kh = blockIdx.y, b = blockIdx.z / a.n_sub, rb = (blockIdx.z % a.n_sub) * a.Rs;
+    const int sp = blockIdx.x, kh = blockIdx.y / a.n_hsplit, b = blockIdx.z / a.n_sub, rb = (blockIdx.z % a.n_sub) * a.Rs;
+    const int h0 = kh * (a.n_q / a.n_kv) + (int)(blockIdx.y % a.n_hsplit) * a.hs;      // first query head of this CTA
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef TASC_TIMELINE
     struct LogAtExit { unsigned long long t0, ta, tb, tc, td, te, tf; __device__ ~LogAtExit() { if (threadIdx.x == 0) ctalog_put(t0, ta, tb, 10, tc, td, te, tf); } } log_at_exit{global_ns(), 0, 0, 0, 0, 0, 0};
 #endif
-    const int g = a.n_q / a.n_kv, R = a.Rs;                   // R: rows of this CTA's sub-block; its first row is rb
+    const int g = a.hs, R = a.Rs;                              // g: query heads of this CTA; R: rows of its sub-block, the first is rb
     const int G = g * R;
     const int qd = a.n_q * HD;
 
@@ -161,7 +165,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int rho = i / (HD / 4), d4 = (i % (HD / 4)) * 4;
                 const int m = b * a.R + rb + rho % R;
                 const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
-                const size_t col = (size_t)(kh * g + rho / R) * HD + d4;
+                const size_t col = (size_t)(h0 + rho / R) * HD + d4;
                 *reinterpret_cast<uint2*>(a.out + row * qd + col) = make_uint2(0u, 0u);
                 *reinterpret_cast<uint2*>(a.out + (row + a.TB) * qd + col) = make_uint2(0u, 0u);
             }
@@ -177,7 +181,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int n_slabs = (G + 15) / 16;
     // A warp owns one 16-row slab of one key tile.  With fewer slabs than warps the warps form ng = 2 or 4 groups
     // of n_slabs warps; group `grp` handles tiles grp, grp + ng, ...; the groups' results are merged in shared memory.
-    const int ng = warp_groups(n_slabs, STAGES);
+    const int ng = warp_groups(n_slabs, STAGES, n_tiles);
     const int slab = warp % n_slabs, grp = warp / n_slabs;
     const bool computes = grp < ng;
     const int n_super = (n_tiles + ng - 1) / ng;                 // iterations of ng tiles
@@ -268,10 +272,10 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             cp_async_commit();                                   // one group per iteration, empty past the end
         }
     };
-    // prologue of the ring: tiles that lie wholly inside the committed prefix start before the wait,
-    // the tiles holding this step's new rows (written by the preceding grid) after it
+    // prologue of the ring (all super_stages slots): iterations that lie wholly inside the committed prefix are
+    // requested before the wait, those holding this step's new rows (written by the preceding grid) after it
     int issued = 0;
-    while (issued < super_stages - 1 && issued < n_super && k_begin + (issued + 1) * ng * TKEYS <= seq_pos0) {
+    while (issued < super_stages && issued < n_super && k_begin + (issued + 1) * ng * TKEYS <= seq_pos0) {
         load_super(issued);
         ++issued;
     }
@@ -292,10 +296,10 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int hl = rho / R, rr = rho % R;
         qv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (rho < G && rr < rows)
-            qv[j] = *reinterpret_cast<const float4*>(a.q + (size_t)(b * a.R + rb + rr) * qd + (size_t)(kh * g + hl) * HD + d4);
+            qv[j] = *reinterpret_cast<const float4*>(a.q + (size_t)(b * a.R + rb + rr) * qd + (size_t)(h0 + hl) * HD + d4);
     }
     // the rest of the ring's prologue (tiles holding this step's new rows), requested while the Q rows are on their way
-    for (; issued < super_stages - 1; ++issued) load_super(issued);   // commits an empty group past the end
+    for (; issued < super_stages; ++issued) load_super(issued);       // past the end: nothing (cp.async: an empty group)
 #pragma unroll
     for (int j = 0; j < NQ; ++j) {
         const int i = tid + j * THREADS;
@@ -323,8 +327,6 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #endif
 
     for (int sup = 0; sup < n_super; ++sup) {
-        if (sup + super_stages - 1 < n_super) load_super(sup + super_stages - 1);
-        else if (!use_tma) cp_async_commit();
         if (use_tma) {                                             // iteration `sup` has landed (bounded wait)
             for (int j = 0; j < ng; ++j)
                 if (sup * ng + j < n_tiles &&
@@ -430,6 +432,9 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
         __syncthreads();
+        // the slot of this iteration is free again: refill it with the iteration super_stages ahead
+        if (sup + super_stages < n_super) load_super(sup + super_stages);
+        else if (!use_tma) cp_async_commit();
     }
 #ifdef TASC_TIMELINE
     log_at_exit.tb = global_ns();
@@ -482,7 +487,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const float inv = (rr < rows) ? (half ? inv1 : inv0) : 0.f;
                 const int m = b * a.R + rb + rr;
                 const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
-                const size_t col = (size_t)(kh * g + hl) * HD + 2 * (lane & 3);
+                const size_t col = (size_t)(h0 + hl) * HD + 2 * (lane & 3);
 #pragma unroll
                 for (int nt = 0; nt < HD / 8; ++nt) {
                     uint32_t h, l;
@@ -553,7 +558,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         const int m = b * a.R + rb + rr;
         const size_t row = (size_t)(m / a.TB) * (2 * a.TB) + (m % a.TB);
-        const size_t col = (size_t)(kh * g + hl) * HD + d4;
+        const size_t col = (size_t)(h0 + hl) * HD + d4;
         uint2 h, l;
         pack_hilo(acc.x, acc.y, h.x, l.x);
         pack_hilo(acc.z, acc.w, h.y, l.y);
@@ -626,7 +631,7 @@ tasc_status launch_inst(const AttnArgs& a, const CUtensorMap& tmK, const CUtenso
     tasc_status pst = prepare_inst<HD, NS>();
     if (pst != TASC_OK) return pst;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)a.splits, (unsigned)a.n_kv, (unsigned)B);
+    cfg.gridDim = dim3((unsigned)a.splits, (unsigned)(a.n_kv * a.n_hsplit), (unsigned)B);
     cfg.blockDim = dim3(256, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -652,40 +657,57 @@ tasc_status launch_inst(const AttnArgs& a, const CUtensorMap& tmK, const CUtenso
 
 int attention_mma_row_pad(int G) { return G <= 64 ? 64 : 128; }
 
-// Key-range splits per (sequence, KV head) (1..8, the CTAs of a cluster) and ring depth, from a small cost model
-// in microseconds: a CTA needs about 2.5 us to start (Q staging, first tiles) plus one tile time per iteration (its warp groups take `ng`
-// tiles per iteration; a shallow ring adds memory stalls), the clusters run in as many waves as the device's
-// cluster occupancy dictates (one straggling cluster costs a whole wave), and splitting adds the cluster
-// exchange and merge (about 4.5 us).
-AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx) {
+// Query heads per CTA, key-range splits per (sequence, head group) (1..8, the CTAs of a cluster) and ring depth, from a
+// small cost model in microseconds: a CTA needs about 2.5 us to start (Q staging, first tiles) plus one tile time per
+// iteration (its warp groups take `ng` tiles per iteration; a shallow ring adds memory stalls), the clusters run in as
+// many waves as the device's cluster occupancy dictates (one straggling cluster costs a whole wave), and splitting
+// adds the cluster exchange and merge.  With few sequences the g query heads that share a KV head are dealt out to
+// several CTAs (each re-reads that head's K/V from L2, which is cheap next to leaving most SMs idle): fewer query rows
+// per CTA mean fewer slabs, so more warp groups work on different key tiles at once.
+AttnPlan plan_attention_mma(int B, int n_kv, int hd, int g, int rows, int max_ctx) {
     // The launch shape is fixed before the lengths are known (and stays fixed in a captured graph): it is chosen
     // for three quarters of the context the cache can hold; shorter ranges leave the last splits idle.
     const int n_tiles = std::max(1, ((max_ctx * 3) / 4 + TKEYS - 1) / TKEYS);
-    const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;       // nw: slabs of the padded query tile (kernel instance)
-    const int max_stages = hd >= 128 ? (nw > 4 ? 4 : 5) : 8;
     // Measured (microseconds): one iteration of a warp group over a 64-key tile, and the time the SM's mma.sync
     // pipes need per tile and 16-row slab when all warps have work (the lower bound once several groups run).
     const float t_tile = hd >= 128 ? 2.0f : (hd >= 64 ? 1.3f : 0.8f);
     const float t_pipe = hd >= 128 ? 0.6f : (hd >= 64 ? 0.3f : 0.15f);
-    AttnPlan best = {1, max_stages};
+    AttnPlan best = {1, 2, g};
     float best_cost = 1e30f;
-    const int depths[2] = {max_stages, max_stages >= 8 ? 4 : 3};
-    for (int di = 0; di < 2; ++di) {
-        const int stages = depths[di];
-        const int ng = warp_groups(n_slabs, stages);
-        for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
-            int fit = fit_any(hd, nw, s, stages);
-            if (fit <= 0) fit = std::max(1, 148 / s);               // no device to ask: assume one CTA per SM
-            const int waves = (B * n_kv + fit - 1) / fit;
-            const int tiles_cta = (n_tiles + s - 1) / s;
-            const int iters = (tiles_cta + ng - 1) / ng;
-            const float stall = di == 0 ? 0.f : 0.25f * t_tile;      // a shallow ring hides less latency
-            const float loop = std::max(iters * (t_tile + stall), tiles_cta * n_slabs * t_pipe);
-            const float merge = s > 1 ? 0.5f + 0.25f * s : 0.f;      // cluster barrier + one round of remote reads
-            // a grid that takes (nearly) every SM keeps the next kernel's CTAs from starting early
-            const float crowd = B * n_kv * s > 128 ? 3.0f : 0.f;
-            const float cost = waves * (2.5f + loop) + merge + crowd;
-            if (cost < best_cost - 1e-6f) { best_cost = cost; best = AttnPlan{s, stages}; }
+    // Candidates: all g heads of a KV head in one CTA; and, for few sequences with 128-wide heads (where one warp needs
+    // 2 us per key tile), the largest share of the heads whose rows still fill a single 16-row slab.  (Measured: on the
+    // 1.5B shape at one sequence 2 of 6 heads per CTA shorten the step by 4 %; 64-wide heads and larger batches lose.)
+    int hs_slab = g;
+    while (hs_slab > 1 && (g % hs_slab || hs_slab * rows > 16)) --hs_slab;
+    const bool may_split = hd >= 128 && B * n_kv <= 4 && hs_slab * rows <= 16;
+    for (int hs = g; hs >= 1; --hs) {
+        if (g % hs) continue;
+        if (hs != g && !(may_split && hs == hs_slab)) continue;
+        const int G = hs * rows;
+        if (G > 128) continue;
+        const int nw = G <= 64 ? 4 : 8, n_slabs = (G + 15) / 16;       // nw: slabs of the padded query tile (kernel instance)
+        const int max_stages = hd >= 128 ? (nw > 4 ? 4 : 5) : 8;
+        const int depths[2] = {max_stages, max_stages >= 8 ? 4 : 3};
+        const int groups = B * n_kv * (g / hs);                       // clusters of the launch
+        for (int di = 0; di < 2; ++di) {
+            const int stages = depths[di];
+            for (int s = 1; s <= 8 && s <= n_tiles; ++s) {
+                int fit = fit_any(hd, nw, s, stages);
+                if (fit <= 0) fit = std::max(1, 148 / s);               // no device to ask: assume one CTA per SM
+                const int waves = (groups + fit - 1) / fit;
+                const int tiles_cta = (n_tiles + s - 1) / s;
+                const int ng = warp_groups(n_slabs, stages, tiles_cta);
+                const int iters = (tiles_cta + ng - 1) / ng;
+                const float stall = di == 0 ? 0.f : 0.25f * t_tile;      // a shallow ring hides less latency
+                const float loop = std::max(iters * (t_tile + stall), tiles_cta * n_slabs * t_pipe);
+                const float merge = s > 1 ? 0.5f + 0.25f * s : 0.f;      // cluster barrier + one round of remote reads
+                // a grid that takes (nearly) every SM keeps the next kernel's CTAs from starting early
+                const float crowd = groups * s > 128 ? 3.0f : 0.f;
+                // every head group re-reads its KV head's keys: L2 traffic, about 0.1 us per extra pass over a tile
+                const float reread = 0.1f * tiles_cta * (float)(g / hs - 1) / (float)std::max(1, g / hs);
+                const float cost = waves * (2.5f + loop) + merge + crowd + reread;
+                if (cost < best_cost - 1e-6f) { best_cost = cost; best = AttnPlan{s, stages, hs}; }
+            }
         }
     }
     return best;
@@ -700,7 +722,9 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
     const int Rs = R <= 16 ? R : 16;
     if (R % Rs) return TASC_EINVAL;
     const int n_sub = R / Rs;
-    const int G = (n_q / n_kv) * Rs;
+    const int g = n_q / n_kv, hs = plan.heads;
+    if (hs < 1 || g % hs) return TASC_EINVAL;
+    const int G = hs * Rs;
     if (G > 128 || (hd != 32 && hd != 64 && hd != 128) || n_splits < 1 || n_splits > 8) return TASC_EINVAL;
     const int GP = attention_mma_row_pad(G);
     AttnArgs a;
@@ -708,6 +732,7 @@ tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages
     a.max_pages = max_pages; a.page_size = page_size; a.n_pages = n_pages;
     a.seq_pos0 = rp.seq_pos0; a.seq_rows = rp.seq_rows;
     a.out = out; a.TB = TB;
+    a.hs = hs; a.n_hsplit = g / hs;
     a.R = R; a.Rs = Rs; a.n_sub = n_sub; a.n_q = n_q; a.n_kv = n_kv; a.splits = n_splits; a.stages = plan.stages;
     a.scale_log2e = 1.4426950408889634f / sqrtf((float)hd);
     a.status = status;

@@ -14,8 +14,11 @@
 // of  lambda_num * c_corp(x) * T_prompt + (lambda_den - lambda_num) * c_prompt(x) * T_corp  in 64-bit
 // integers with the smallest token id winning ties.
 #include "kernels.h"
+#include "ngram_table.cuh"
 
 #include <algorithm>
+#include <cmath>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -48,69 +51,6 @@ struct tasc_drafter {
 
 namespace tasc {
 namespace {
-
-constexpr uint64_t VALID_BIT = 1ull << 63;
-constexpr int TOK_BITS = TASC_VOCAB_BITS;
-constexpr uint32_t TOK_MASK = (1u << TOK_BITS) - 1u;
-
-struct Key { uint64_t lo, hi; };
-
-// Field j (20 bits) at bit 20*j of the 128-bit word; the order in bits 120..122; bit 127 marks a used slot.
-__host__ __device__ __forceinline__ void key_put(Key& k, int field, uint32_t tok) {
-    const int bit = field * TOK_BITS;
-    const uint64_t v = tok & TOK_MASK;
-    if (bit + TOK_BITS <= 64) k.lo |= v << bit;
-    else if (bit >= 64) k.hi |= v << (bit - 64);
-    else { k.lo |= v << bit; k.hi |= v >> (64 - bit); }
-}
-__host__ __device__ __forceinline__ uint32_t key_get(const Key& k, int field) {
-    const int bit = field * TOK_BITS;
-    uint64_t v;
-    if (bit + TOK_BITS <= 64) v = k.lo >> bit;
-    else if (bit >= 64) v = k.hi >> (bit - 64);
-    else v = (k.lo >> bit) | (k.hi << (64 - bit));
-    return (uint32_t)v & TOK_MASK;
-}
-__host__ __device__ __forceinline__ Key key_make(int n) {
-    Key k;
-    k.lo = 0;
-    k.hi = VALID_BIT | ((uint64_t)n << 56);
-    return k;
-}
-__host__ __device__ __forceinline__ uint64_t key_hash(const Key& k) {
-    uint64_t h = k.lo * 0x9E3779B97F4A7C15ull ^ (k.hi + 0xD6E8FEB86659FD93ull);
-    h ^= h >> 32; h *= 0xD6E8FEB86659FD93ull;
-    h ^= h >> 29; h *= 0x9E3779B97F4A7C15ull;
-    h ^= h >> 32;
-    return h;
-}
-
-// 128-bit compare-and-swap on a 16-byte aligned slot; returns the previous contents.
-__device__ __forceinline__ Key cas128(uint64_t* addr, Key cmp, Key val) {
-    Key old;
-    asm volatile(
-        "{\n\t.reg .b128 c, n, o;\n\t"
-        "mov.b128 c, {%2, %3};\n\t"
-        "mov.b128 n, {%4, %5};\n\t"
-        "atom.global.cas.b128 o, [%6], c, n;\n\t"
-        "mov.b128 {%0, %1}, o;\n\t}"
-        : "=l"(old.lo), "=l"(old.hi)
-        : "l"(cmp.lo), "l"(cmp.hi), "l"(val.lo), "l"(val.hi), "l"(addr)
-        : "memory");
-    return old;
-}
-
-// Claim or find the slot of `key`; returns the slot or ~0 when the table is full.
-__device__ __forceinline__ uint64_t table_upsert(uint64_t* keys, uint64_t mask, Key key) {
-    uint64_t slot = key_hash(key) & mask;
-    const Key empty = {0ull, 0ull};
-    for (uint64_t probe = 0; probe <= mask; ++probe) {
-        const Key old = cas128(keys + 2 * slot, empty, key);
-        if ((old.lo == 0 && old.hi == 0) || (old.lo == key.lo && old.hi == key.hi)) return slot;
-        slot = (slot + 1) & mask;
-    }
-    return ~0ull;
-}
 
 // remaining[i] = number of tokens after position i inside its document, clamped to 255
 __global__ void mark_remaining_kernel(const int64_t* __restrict__ offsets, int64_t n_docs, int64_t T, uint8_t* remaining) {
@@ -196,6 +136,157 @@ __global__ void succ_fill_kernel(const uint64_t* __restrict__ skeys, const uint3
     s.next = (int32_t)key_get(e, n);
     s.count = counts[i];
     t.succ[pos] = s;
+}
+
+
+// Order-1 model with one successor of count 1 per context: context token c -> table[c].
+__global__ void bigram_insert_kernel(const int32_t* __restrict__ table, int vocab, OrderTable t, int* status) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= vocab) return;
+    const int x = table[c];
+    if (x < 0 || x >= vocab) { set_status(status, TASC_EINVAL); return; }
+    Key key = key_make(1);
+    key_put(key, 0, (uint32_t)c);
+    const uint64_t slot = table_upsert(t.keys, t.mask, key);
+    if (slot == ~0ull) { set_status(status, TASC_ECAPACITY); return; }
+    CtxVal v;
+    v.offset = (unsigned long long)c; v.n_succ = 1u; v.total = 1u;
+    t.vals[slot] = v;
+    Succ sc;
+    sc.next = x; sc.count = 1u;
+    t.succ[c] = sc;
+}
+
+// ------------------------------------------------------------------------------------------- corpus statistics
+// The statistics are functions of the multiset of counts only, so the device first turns the count table into a
+// histogram of count VALUES (how many bigrams occur c times), which is exact integer work whose result does not
+// depend on where the hash table put anything; one block then walks that histogram in a fixed order.
+constexpr int CC_BITS = 20;                       // count values below 2^20 have a histogram bin of their own
+constexpr uint32_t CC_BINS = 1u << CC_BITS;
+constexpr int CC_OVERFLOW = 4096;                 // larger count values are listed individually
+constexpr int STATS_THREADS = 1024;
+
+// [0] distinct keys, [1] overflow entries, [2] sum of squared counts
+__global__ void count_values_kernel(const uint32_t* __restrict__ counts, uint64_t n, uint32_t* __restrict__ bins,
+                                    uint32_t* __restrict__ overflow, unsigned long long* __restrict__ scal, int* status) {
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t c = i < n ? counts[i] : 0u;
+    unsigned long long sq = (unsigned long long)c * c;
+    unsigned int nz = c ? 1u : 0u;
+    if (c) {
+        if (c < CC_BINS) atomicAdd(&bins[c], 1u);
+        else {
+            const unsigned long long at = atomicAdd(&scal[1], 1ull);
+            if (at < CC_OVERFLOW) overflow[at] = c; else set_status(status, TASC_ECAPACITY);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
+        nz += __shfl_xor_sync(0xFFFFFFFFu, nz, o);
+    }
+    if ((threadIdx.x & 31) == 0 && nz) {
+        atomicAdd(&scal[0], (unsigned long long)nz);
+        atomicAdd(&scal[2], sq);                   // integer sums: the order of the additions does not matter
+    }
+}
+
+struct CountSummary {
+    unsigned long long n_total;      // sum of the counts
+    unsigned long long n_distinct;
+    unsigned long long sum_sq;
+    unsigned long long n_for_cdf;    // smallest number of the largest counts that reach cdf_num / cdf_den of n_total
+    double sum_c_log2_c;             // sum over all keys of c log2 c
+};
+
+// One block.  bins[c] = number of keys with count c (c < 2^20), overflow[] = the counts >= 2^20.  Walks the count
+// values from the largest down: thread t owns a contiguous range of bins, an exclusive scan over the threads
+// gives the mass and the number of keys above its range, and the thread whose range holds the crossing of the
+// coverage target finishes the count by itself.  Sums are taken in a fixed order, so the result is reproducible.
+__global__ void __launch_bounds__(STATS_THREADS)
+count_summary_kernel(const uint32_t* __restrict__ bins, uint32_t* __restrict__ overflow, const unsigned long long* __restrict__ scal,
+                     unsigned long long cdf_num, unsigned long long cdf_den, CountSummary* out) {
+    __shared__ unsigned long long s_mass[STATS_THREADS], s_keys[STATS_THREADS];
+    __shared__ double s_log[STATS_THREADS];
+    __shared__ uint32_t s_over[CC_OVERFLOW];
+    __shared__ unsigned long long s_result, s_over_mass;
+    __shared__ double s_over_log;
+    const int t = threadIdx.x;
+    const int n_over = (int)min(scal[1], (unsigned long long)CC_OVERFLOW);
+    // the overflow list, largest first: rank by counting (a few thousand entries at most)
+    for (int i = t; i < n_over; i += STATS_THREADS) {
+        const uint32_t c = overflow[i];
+        int rank = 0;
+        for (int j = 0; j < n_over; ++j) {
+            const uint32_t o = overflow[j];
+            rank += (o > c || (o == c && j < i)) ? 1 : 0;
+        }
+        s_over[rank] = c;
+    }
+    __syncthreads();
+    if (t == 0) {
+        unsigned long long m = 0;
+        double l = 0.0;
+        for (int i = 0; i < n_over; ++i) { m += s_over[i]; l += (double)s_over[i] * log2((double)s_over[i]); }
+        s_over_mass = m; s_over_log = l; s_result = 0ull;
+    }
+    // thread t owns bins hi, hi - 1, ..., lo (descending count values)
+    constexpr uint32_t PER = CC_BINS / STATS_THREADS;
+    const uint32_t hi = CC_BINS - 1u - (uint32_t)t * PER, lo = hi - (PER - 1u);
+    unsigned long long mass = 0, keys = 0;
+    double lg = 0.0;
+    for (uint32_t c = hi; ; --c) {
+        const uint32_t m = c ? bins[c] : 0u;
+        if (m) { mass += (unsigned long long)m * c; keys += m; lg += (double)m * ((double)c * log2((double)c)); }
+        if (c == lo) break;
+    }
+    s_mass[t] = mass; s_keys[t] = keys; s_log[t] = lg;
+    __syncthreads();
+    if (t == 0) {
+        // serial exclusive scan over the 1,024 partial sums (fixed order)
+        unsigned long long m = s_over_mass, k = (unsigned long long)n_over;
+        double l = s_over_log;
+        for (int i = 0; i < STATS_THREADS; ++i) {
+            const unsigned long long mi = s_mass[i], ki = s_keys[i];
+            l += s_log[i];
+            s_mass[i] = m; s_keys[i] = k;
+            m += mi; k += ki;
+        }
+        out->n_total = m; out->n_distinct = k; out->sum_sq = scal[2]; out->sum_c_log2_c = l;
+        s_over_mass = m;                                     // total mass, for the threads below
+    }
+    __syncthreads();
+    const unsigned long long total = s_over_mass;
+    if (total == 0) { if (t == 0) out->n_for_cdf = 0; return; }
+    // target: smallest run with run * den >= num * total.  128-bit products are not needed: total < 2^40, num, den <= 2^16.
+    const unsigned long long need = (cdf_num * total + cdf_den - 1) / cdf_den;
+    if (t == 0) {
+        // crossing inside the overflow list?
+        unsigned long long run = 0;
+        for (int i = 0; i < n_over; ++i) {
+            run += s_over[i];
+            if (run >= need) { s_result = (unsigned long long)i + 1; break; }
+        }
+    }
+    __syncthreads();
+    const unsigned long long above = s_mass[t];
+    if (s_result == 0 && above < need && above + mass >= need) {
+        unsigned long long run = above, k = s_keys[t];
+        for (uint32_t c = hi; ; --c) {
+            const uint32_t m = c ? bins[c] : 0u;
+            if (m) {
+                if (run + (unsigned long long)m * c >= need) {
+                    k += (need - run + c - 1) / c;
+                    break;
+                }
+                run += (unsigned long long)m * c; k += m;
+            }
+            if (c == lo) break;
+        }
+        s_result = k;
+    }
+    __syncthreads();
+    if (t == 0) out->n_for_cdf = s_result;
 }
 
 // ------------------------------------------------------------------------------------------- draft
@@ -388,14 +479,6 @@ void free_tables(DeviceTables& dt) {
     }
 }
 
-uint64_t pow2_at_least(uint64_t v) {
-    uint64_t p = 64;
-    while (p < v) p <<= 1;
-    return p;
-}
-
-inline unsigned blocks_for(uint64_t n, int threads) { return (unsigned)((n + threads - 1) / threads); }
-
 }  // namespace
 }  // namespace tasc
 
@@ -518,6 +601,128 @@ extern "C" tasc_status tasc_drafter_build(const int32_t* corpus_tokens, const in
     return TASC_OK;
 }
 
+extern "C" tasc_status tasc_drafter_from_bigram(const int32_t* table, int32_t vocab, tasc_stream stream_, tasc_drafter** out) {
+    if (!out) return TASC_EINVAL;
+    *out = nullptr;
+    if (!table || vocab < 1 || vocab > (1 << TASC_VOCAB_BITS)) return TASC_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    tasc_drafter* d = new (std::nothrow) tasc_drafter();
+    if (!d) return TASC_ENOMEM;
+    for (int n = 0; n <= TASC_MAX_ORDER; ++n) d->dt.t[n] = OrderTable{nullptr, nullptr, nullptr, 0, 0};
+    d->dt.n_max = 1; d->dt.fallback = 0; d->p_min = 1; d->vocab = vocab;
+    cudaGetDevice(&d->device);
+    OrderTable& t = d->dt.t[1];
+    const uint64_t cap = pow2_at_least(2 * (uint64_t)vocab);
+    t.mask = cap - 1;
+    t.n_succ = vocab;
+    int* status = nullptr;
+    tasc_status rc = TASC_OK;
+    if (cudaMalloc(reinterpret_cast<void**>(&t.keys), cap * 16) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&t.vals), cap * sizeof(CtxVal)) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&t.succ), (size_t)vocab * sizeof(Succ)) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&status), sizeof(int)) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ENOMEM; }
+    if (rc == TASC_OK) {
+        cudaMemsetAsync(t.keys, 0, cap * 16, stream);
+        cudaMemsetAsync(t.vals, 0, cap * sizeof(CtxVal), stream);
+        cudaMemsetAsync(status, 0, sizeof(int), stream);
+        bigram_insert_kernel<<<blocks_for((uint64_t)vocab, 256), 256, 0, stream>>>(table, vocab, t, status);
+        int st = 0;
+        if (cudaMemcpyAsync(&st, status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ECUDA; }
+        else if (st != 0) rc = st;
+    }
+    if (status) cudaFree(status);
+    if (rc != TASC_OK) {
+        free_tables(d->dt);
+        delete d;
+        return rc;
+    }
+    *out = d;
+    return TASC_OK;
+}
+
+extern "C" tasc_status tasc_corpus_stats(const int32_t* corpus_tokens, const int64_t* doc_offsets, int64_t n_docs, int32_t vocab,
+                                         int32_t cdf_num, int32_t cdf_den, tasc_stream stream_, tasc_corpus_statistics* out) {
+    if (!out || !doc_offsets || n_docs < 0 || vocab < 1 || vocab > (1 << TASC_VOCAB_BITS) || cdf_den < 1 || cdf_den > 65536 ||
+        cdf_num < 1 || cdf_num > cdf_den)
+        return TASC_EINVAL;
+    *out = tasc_corpus_statistics{};
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    std::vector<int64_t> offs((size_t)n_docs + 1);
+    TASC_CUDA_TRY(cudaMemcpyAsync(offs.data(), doc_offsets, offs.size() * sizeof(int64_t), cudaMemcpyDeviceToHost, stream));
+    TASC_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (offs[0] != 0) return TASC_EINVAL;
+    uint64_t pairs = 0;
+    for (int64_t d = 0; d < n_docs; ++d) {
+        const int64_t len = offs[d + 1] - offs[d];
+        if (len < 0) return TASC_EINVAL;
+        pairs += (uint64_t)std::max<int64_t>(0, len - 1);
+    }
+    const int64_t T = offs[n_docs];
+    if (T > 0 && !corpus_tokens) return TASC_EINVAL;
+    if ((uint64_t)T >= (1ull << 40)) return TASC_EINVAL;
+
+    uint8_t* remaining = nullptr;
+    uint32_t *hist = nullptr, *bins = nullptr, *overflow = nullptr, *scounts = nullptr;
+    unsigned long long* scal = nullptr;      // [0..2] bigram scalars, [4..6] token scalars
+    CountSummary* summ = nullptr;            // [0] bigrams, [1] tokens
+    int* status = nullptr;
+    uint64_t* skeys = nullptr;
+    const uint64_t cap = pow2_at_least(2 * std::max<uint64_t>(pairs, 1));
+    tasc_status rc = TASC_OK;
+#define TRY_ALLOC(ptr, bytes) if (rc == TASC_OK && cudaMalloc(reinterpret_cast<void**>(&(ptr)), (bytes)) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ENOMEM; }
+    TRY_ALLOC(remaining, (size_t)std::max<int64_t>(T, 1));
+    TRY_ALLOC(hist, (size_t)vocab * sizeof(uint32_t));
+    TRY_ALLOC(bins, 2 * (size_t)CC_BINS * sizeof(uint32_t));
+    TRY_ALLOC(overflow, 2 * (size_t)CC_OVERFLOW * sizeof(uint32_t));
+    TRY_ALLOC(scal, 8 * sizeof(unsigned long long));
+    TRY_ALLOC(summ, 2 * sizeof(CountSummary));
+    TRY_ALLOC(status, sizeof(int));
+    TRY_ALLOC(skeys, cap * 16);
+    TRY_ALLOC(scounts, cap * 4);
+#undef TRY_ALLOC
+    CountSummary h[2] = {};
+    if (rc == TASC_OK) {
+        cudaMemsetAsync(hist, 0, (size_t)vocab * sizeof(uint32_t), stream);
+        cudaMemsetAsync(bins, 0, 2 * (size_t)CC_BINS * sizeof(uint32_t), stream);
+        cudaMemsetAsync(scal, 0, 8 * sizeof(unsigned long long), stream);
+        cudaMemsetAsync(status, 0, sizeof(int), stream);
+        cudaMemsetAsync(skeys, 0, cap * 16, stream);
+        cudaMemsetAsync(scounts, 0, cap * 4, stream);
+        if (T > 0) {
+            mark_remaining_kernel<<<blocks_for(T, 256), 256, 0, stream>>>(doc_offsets, n_docs, T, remaining);
+            token_hist_kernel<<<blocks_for(T, 256), 256, 0, stream>>>(corpus_tokens, T, vocab, hist, status);
+            // bigrams = the windows of the order-1 model before pruning: (token, next) inside one document
+            count_kernel<<<blocks_for(T, 256), 256, 0, stream>>>(corpus_tokens, remaining, T, 1, skeys, scounts, cap - 1, status);
+        }
+        count_values_kernel<<<blocks_for(cap, 256), 256, 0, stream>>>(scounts, cap, bins, overflow, scal, status);
+        count_values_kernel<<<blocks_for(vocab, 256), 256, 0, stream>>>(hist, (uint64_t)vocab, bins + CC_BINS, overflow + CC_OVERFLOW, scal + 4, status);
+        count_summary_kernel<<<1, STATS_THREADS, 0, stream>>>(bins, overflow, scal, (unsigned long long)cdf_num, (unsigned long long)cdf_den, summ);
+        count_summary_kernel<<<1, STATS_THREADS, 0, stream>>>(bins + CC_BINS, overflow + CC_OVERFLOW, scal + 4, 1ull, 1ull, summ + 1);
+        int st = 0;
+        if (cudaMemcpyAsync(h, summ, sizeof(h), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+            cudaMemcpyAsync(&st, status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ECUDA; }
+        else if (st != 0) rc = st;
+    }
+    cudaFree(remaining); cudaFree(hist); cudaFree(bins); cudaFree(overflow); cudaFree(scal); cudaFree(summ);
+    cudaFree(status); cudaFree(skeys); cudaFree(scounts);
+    if (rc != TASC_OK) return rc;
+    // the closing arithmetic on a handful of scalars: H = log2 N - (sum c log2 c) / N;  H_2 = 2 log2 N - log2 sum c^2
+    auto entropy = [](const CountSummary& c) { return c.n_total ? log2((double)c.n_total) - c.sum_c_log2_c / (double)c.n_total : 0.0; };
+    out->n_tokens = T;
+    out->n_bigrams = (int64_t)h[0].n_total;
+    out->n_unique_tokens = (int64_t)h[1].n_distinct;
+    out->n_unique_bigrams = (int64_t)h[0].n_distinct;
+    out->bigrams_for_cdf = (int64_t)h[0].n_for_cdf;
+    out->bigram_entropy_bits = entropy(h[0]);
+    out->typical_set_size = exp2(out->bigram_entropy_bits);
+    out->token_entropy_bits = entropy(h[1]);
+    out->token_entropy_normalised = vocab > 1 ? out->token_entropy_bits / log2((double)vocab) : 0.0;
+    out->token_renyi2_bits = h[1].n_total ? 2.0 * log2((double)h[1].n_total) - log2((double)h[1].sum_sq) : 0.0;
+    return TASC_OK;
+}
+
 extern "C" tasc_status tasc_drafter_export(const tasc_drafter* d, tasc_ngram_entry* out, int64_t cap, int64_t* n_entries,
                                            int32_t* fallback_token) {
     if (!d || !n_entries || cap < 0 || (cap > 0 && !out)) return TASC_EINVAL;
@@ -576,10 +781,18 @@ extern "C" tasc_status tasc_draft(const tasc_drafter* d, const int32_t* tokens, 
     uint64_t hs = 64;
     while (hs * 3 < (uint64_t)stride * 4) hs <<= 1;      // load factor <= 3/4
     const size_t smem = hs * 8 + (size_t)stride * sizeof(int32_t);      // hash of the context successors + the tokens
-    static bool attr = false;
-    if (!attr) {
-        TASC_CUDA_TRY(cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 184 * 1024));
-        attr = true;
+    {
+        // the attribute belongs to the device: set once per device, under a lock (two threads may make their first call together)
+        static std::mutex mu;
+        static bool attr_done[64] = {false};
+        int dev = 0;
+        TASC_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return TASC_EINVAL;
+        std::lock_guard<std::mutex> lk(mu);
+        if (!attr_done[dev]) {
+            TASC_CUDA_TRY(cudaFuncSetAttribute(draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 184 * 1024));
+            attr_done[dev] = true;
+        }
     }
     ProfScope ps(K_DRAFT, static_cast<cudaStream_t>(stream));
     draft_kernel<<<B, DRAFT_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(

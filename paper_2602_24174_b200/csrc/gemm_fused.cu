@@ -620,9 +620,9 @@ tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const Fus
 
 }  // namespace
 
-FusedPlan plan_fused(int M, int N, int K, int epi) {
+FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles) {
     FusedPlan p;
-    p.TBL = gemm_token_tile(M, true);
+    p.TBL = gemm_token_tile(M, true, few_tiles);
     // The LM head streams the largest matrix once and has no split-K exchange: one CTA takes as many layout tiles
     // as an MMA holds (256 columns), so that a weight tile is fetched by one CTA, not by one per token tile.
     const int span = epi == EPI_LM ? std::max(1, std::min((M + p.TBL - 1) / p.TBL, 128 / p.TBL)) : 1;

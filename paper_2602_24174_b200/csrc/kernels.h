@@ -32,7 +32,8 @@ struct GemmPlan {
     int smem_bytes;
 };
 GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes, bool pair);
-int gemm_token_tile(int M, bool pair);     // TB for M token rows
+// TB for M token rows.  few_tiles (1..3): how many token tiles 49..128 paired rows are cut into at least (see gemm_token_tile).
+int gemm_token_tile(int M, bool pair, int few_tiles = 3);
 inline size_t gemm_partial_bytes(const GemmPlan& p, int M, int N) { return (size_t)p.splits * M * N * sizeof(float); }
 
 // rows x cols bf16 row-major matrix, box = {64 cols, box_rows}, 128-byte swizzle.
@@ -85,7 +86,7 @@ struct FusedPlan {
     int S;             // cluster size = k-splits
     int stages, data_bytes, smem_bytes;
 };
-FusedPlan plan_fused(int M, int N, int K, int epi);
+FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles = 3);
 // tmW: weight map with box rows 128 (64 for EPI_SWIGLU); tmX: (hi, lo) activation map with box rows BN = 2 TB.
 tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
                               cudaStream_t stream);
@@ -152,6 +153,9 @@ void launch_forced_targets(int mode, const int32_t* drafts, const int32_t* conti
 void launch_gather_output(const int32_t* tokens, int64_t stride, const int32_t* prompt_len, int B, int max_new,
                           int32_t* out, cudaStream_t stream);
 void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, int* out_min, cudaStream_t stream);
+// Model-derived bigram table: B single-token sequences t0 .. t0 + B - 1, and table[t0 + b] = argmax of row b.
+void launch_bigram_rows(int32_t* tokens, int32_t* len, int t0, int vocab, int B, cudaStream_t stream);
+void launch_bigram_store(const unsigned long long* argmax, int32_t* table, int t0, int vocab, int B, cudaStream_t stream);
 
 // ------------------------------------------------------------------ attention (attention.cu)
 // Verify attention of R query rows per sequence over the paged KV cache (grouped-query, causal within the rows).
@@ -165,14 +169,16 @@ int attention_splits(int B, int n_kv, int max_ctx);
 
 // ------------------------------------------------------------------ tensor-core attention for bf16 models (attention_mma.cu)
 struct AttnPlan {
-    int splits;      // key-range splits per (sequence, KV head) = cluster size, 1..8
+    int splits;      // key-range splits per (sequence, head group) = cluster size, 1..8
     int stages;      // depth of the K/V tile ring
+    int heads;       // query heads per CTA: a divisor of n_q / n_kv (the heads sharing a KV head are dealt out to several CTAs)
 };
 // Same contract as launch_attention; the result goes to `out` as (hi, lo) bf16 rows; needs no scratch memory.
 tasc_status launch_attention_mma(const float* qbuf, const __nv_bfloat16* k_pages, const __nv_bfloat16* v_pages,
                                  const int32_t* block_table, int max_pages, int page_size, long long n_pages,
                                  const RowPlan& rp, __nv_bfloat16* out, int TB, int B, int R, int n_q, int n_kv, int hd,
                                  const AttnPlan& plan, int* status, cudaStream_t stream);
-AttnPlan plan_attention_mma(int B, int n_kv, int hd, int G, int max_ctx);
+// B sequences (or sequence blocks), g = n_q / n_kv query heads per KV head, `rows` query rows per sequence block
+AttnPlan plan_attention_mma(int B, int n_kv, int hd, int g, int rows, int max_ctx);
 
 }  // namespace tasc

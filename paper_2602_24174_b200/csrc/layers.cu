@@ -315,6 +315,19 @@ __global__ void forced_targets_kernel(int mode, const int32_t* drafts, const int
     targets[t] = v;
 }
 
+// Single-token contexts t0, t0 + 1, ... as B sequences of length one (ids past the vocabulary repeat the last token).
+__global__ void bigram_rows_kernel(int32_t* tokens, int32_t* len, int t0, int vocab, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    tokens[b] = min(t0 + b, vocab - 1);
+    len[b] = 1;
+}
+__global__ void bigram_store_kernel(const unsigned long long* __restrict__ argmax, int32_t* table, int t0, int vocab, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B || t0 + b >= vocab) return;
+    table[t0 + b] = (int32_t)packed_id(argmax[b]);
+}
+
 __global__ void gather_output_kernel(const int32_t* tokens, int64_t stride, const int32_t* prompt_len, int B, int max_new,
                                      int32_t* out) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -425,6 +438,14 @@ void launch_gather_output(const int32_t* tokens, int64_t stride, const int32_t* 
     ProfScope ps(K_OTHER, stream);
     const int n = B * max_new;
     gather_output_kernel<<<(n + 255) / 256, 256, 0, stream>>>(tokens, stride, prompt_len, B, max_new, out);
+}
+void launch_bigram_rows(int32_t* tokens, int32_t* len, int t0, int vocab, int B, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
+    bigram_rows_kernel<<<(B + 127) / 128, 128, 0, stream>>>(tokens, len, t0, vocab, B);
+}
+void launch_bigram_store(const unsigned long long* argmax, int32_t* table, int t0, int vocab, int B, cudaStream_t stream) {
+    ProfScope ps(K_OTHER, stream);
+    bigram_store_kernel<<<(B + 127) / 128, 128, 0, stream>>>(argmax, table, t0, vocab, B);
 }
 void launch_min_generated(const int32_t* len, const int32_t* prompt_len, int B, int* out_min, cudaStream_t stream) {
     ProfScope ps(K_OTHER, stream);

@@ -90,7 +90,9 @@ def main():
     base = t0.min()
     us = lambda a: (a - base) / 1e3
     kernels, cur = [], None
-    for i in np.argsort(t0):                         # consecutive kernels of the chain have different tags
+    # a CTA leaves only after its grid's predecessor has finished, so end times (not start times: grids start ahead of
+    # one another) separate the kernels of the chain; consecutive kernels have different tags
+    for i in np.argsort(t1):
         if cur is None or tag[i] != cur[0]:
             cur = (int(tag[i]), [])
             kernels.append(cur)
@@ -105,6 +107,7 @@ def main():
         a = agg[NAMES.get(tg, str(tg))]
         a["n"] += 1; a["ctas"] += len(ix)
         a["period"] += end - us(prev_end); a["lag"] += wait - us(prev_end); a["main"] += acc - wait; a["tail"] += end - acc
+        a["lead_first"] += us(prev_end) - us(t0[ix].min()); a["lead_last"] += us(prev_end) - us(t0[ix].max())
         st = [us(x[ix].max()) for x in tx]
         if tg == 10:
             a["p0"] += st[0] - wait; a["p1"] += st[1] - st[0]; a["p2"] += acc - st[1]
@@ -119,9 +122,10 @@ def main():
         else:
             det = (f"tail: TMEM->smem {a['p0']/c:.2f}, cluster barrier {a['p1']/c:.2f}, split-K pull {a['p2']/c:.2f}, "
                    f"epilogue {a['p3']/c:.2f}, leave {a['p4']/c:.2f}")
-        print(f"{name:7s} {int(c):3d} {int(a['ctas']/c):5d} | {a['period']/c:6.2f} = {a['lag']/c:5.2f} + {a['main']/c:5.2f} + {a['tail']/c:5.2f} | {det}")
+        print(f"{name:7s} {int(c):3d} {int(a['ctas']/c):5d} | {a['period']/c:6.2f} = {a['lag']/c:5.2f} + {a['main']/c:5.2f} + {a['tail']/c:5.2f} | "
+              f"started {a['lead_first']/c:.1f} .. {a['lead_last']/c:.1f} before | {det}")
     print("wait lag: predecessor's end -> last CTA past griddepcontrol.wait; main: -> accumulator complete (GEMM) / key tiles done "
-          "(attention); tail: -> last CTA gone")
+          "(attention); tail: -> last CTA gone; started: first .. last CTA start, microseconds before the predecessor's end")
 
 
 if __name__ == "__main__":

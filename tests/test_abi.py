@@ -39,14 +39,15 @@ def test_library_exports_every_declared_symbol(lib_path):
 
 def test_struct_sizes_match_c(lib_path, tmp_path):
     src = tmp_path / "sizes.c"
-    src.write_text('#include <stdio.h>\n#include "tasc.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n",'
+    src.write_text('#include <stdio.h>\n#include "tasc.h"\nint main(void){printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu\\n",'
                    "sizeof(tasc_ngram_entry),sizeof(tasc_model_desc),sizeof(tasc_weights),sizeof(tasc_kv),"
-                   "sizeof(tasc_seqs),sizeof(tasc_draft_params),sizeof(tasc_stats),sizeof(tasc_status));return 0;}\n")
+                   "sizeof(tasc_seqs),sizeof(tasc_draft_params),sizeof(tasc_stats),sizeof(tasc_status),"
+                   "sizeof(tasc_corpus_statistics));return 0;}\n")
     exe = tmp_path / "sizes"
     subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     sizes = list(map(int, subprocess.check_output([str(exe)]).split()))
     from paper_2602_24174_b200 import binding as b
-    mirrors = [b.NgramEntry, b.ModelDesc, b.Weights, b.Kv, b.Seqs, b.DraftParams, b.Stats, ctypes.c_int32]
+    mirrors = [b.NgramEntry, b.ModelDesc, b.Weights, b.Kv, b.Seqs, b.DraftParams, b.Stats, ctypes.c_int32, b.CorpusStatistics]
     assert sizes == [ctypes.sizeof(m) for m in mirrors]
 
 
@@ -61,5 +62,7 @@ def test_argument_checks_need_no_device(lib_path):
     h = ctypes.c_void_p()
     assert b.lib.tasc_drafter_build(None, None, 0, 3, 1, 10, None, ctypes.byref(h)) == b.EINVAL
     assert b.lib.tasc_model_create(None, None, ctypes.byref(h)) == b.EINVAL
+    st = b.CorpusStatistics()
+    assert b.lib.tasc_corpus_stats(None, None, 0, 10, 4, 5, None, ctypes.byref(st)) == b.EINVAL
     assert b.lib.tasc_gemm_workspace_bytes(0, 1, 1) == 0
     assert b.lib.tasc_gemm_workspace_bytes(6, 1152, 896) >= 6 * 1152 * 4
