@@ -140,3 +140,25 @@ def test_drafts_do_not_depend_on_table_layout():
         tok[i, :len(c)] = c; ln[i] = len(c)
     t, l = torch.from_numpy(tok).cuda(), torch.from_numpy(ln).cuda()
     assert torch.equal(b.tasc_draft(dr1, t, l, 4), b.tasc_draft(dr2, t, l, 4))
+
+
+@pytest.mark.gpu
+def test_config2_full_corpus_tables():
+    """All 200,000 documents (14 M tokens) of configuration 2's corpus, n_max 4, p_min 5: export bit-exact."""
+    cfg = configs.get(2)
+    tokens, offsets = corpus.make_corpus(cfg)
+    assert len(offsets) - 1 == 200000
+    b, dr, ng = build_both(tokens, offsets, cfg.n_max, cfg.p_min, cfg.model.vocab)
+    assert_tables_equal(dr, ng)
+
+
+@pytest.mark.gpu
+def test_config4_corpus_slice_tables_at_order_5():
+    """The first 200,000 of configuration 4's 1,000,000 documents (22 M tokens, 110 M count updates at n_max 5,
+    the 20,000-phrase pool): the largest slice the sort-based oracle builder handles in about two minutes."""
+    cfg = configs.get(4)
+    tokens, offsets = corpus.make_corpus(cfg, n_docs=200000)
+    b, dr, ng = build_both(tokens, offsets, cfg.n_max, cfg.p_min, cfg.model.vocab)
+    assert_tables_equal(dr, ng)
+    ctxs = draft_contexts(cfg, tokens, offsets, 24, 600, seed=4)
+    assert_drafts_equal(b, dr, ng, ctxs, cfg.k, [(3, 4), (1, 1)], stride=640)

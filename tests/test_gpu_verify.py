@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from oracle import decode as G
-from tests.gpu_harness import lockstep, make_setup, need_gpu
+from tests.gpu_harness import lockstep, make_setup, need_gpu, record_parity
 from workload import configs, corpus
 
 # logits tolerance: float32 model 1e-4 absolute; bf16 models max-abs 2e-2 / relative 1e-2.
@@ -14,14 +14,37 @@ F32_TOL = dict(logit_atol=1e-4, logit_rtol=0.0, gap_tol=2e-4)
 BF16_TOL = dict(logit_atol=2e-2, logit_rtol=1e-2, gap_tol=1e-2)
 
 
-def check(rep, max_near_tie_frac=0.25):
+def check(rep, name, max_near_tie_frac=0.05):
+    """Drafts bit-exact, no logit outside the tolerance, no argmax mismatch outside a near-tie, and near-tie
+    mismatches on at most 5 % of the compared rows (observed: below 1 %); the counts go to the parity report."""
+    record_parity(name, rep)
+    print(f"lockstep {name}: steps={rep.steps} rows={rep.rows} near_tie_mismatches={rep.near_tie_mismatches} "
+          f"max_logit_err={rep.max_logit_err:.3e} (x{rep.max_err_over_or_bound:.2f} of the either-bound reading)")
     assert rep.steps > 0
     assert rep.draft_mismatches == 0, "drafts must be bit-exact"
     assert not rep.hard_mismatches, rep.hard_mismatches[:5]
     assert rep.accept_mismatches == 0
-    assert rep.near_tie_mismatches <= max_near_tie_frac * rep.rows
-    print(f"lockstep: steps={rep.steps} rows={rep.rows} near_tie_mismatches={rep.near_tie_mismatches} "
-          f"max_logit_err={rep.max_logit_err:.3e}")
+    assert rep.near_tie_mismatches <= max(1, max_near_tie_frac * rep.rows)
+
+
+def assert_diverges_only_at_a_near_tie(got, spec, gap_tol, what):
+    """A free-running generation may leave the oracle's only at a token whose own logit row had a top-2 gap below
+    the tolerance in the oracle (the row that produced the first differing token, not any row anywhere)."""
+    want = np.array(spec.tokens)
+    if np.array_equal(got, want):
+        return None
+    first = int(np.argmax(got != want))
+    # the oracle step and row that produced generated token `first`: a step commits its accepted drafts
+    # (rows 0..a-1 confirmed them) and then the argmax of row a
+    g = 0
+    for st in spec.steps:
+        n = st.n_accepted + 1
+        if first < g + n:
+            row = first - g
+            assert st.gap[row] < gap_tol, f"{what} diverges at token {first} (row {row}, gap {st.gap[row]:.3e}) without a near-tie"
+            return first
+        g += n
+    raise AssertionError(f"{what}: token {first} is beyond the oracle's steps")
 
 
 @pytest.mark.gpu
@@ -29,7 +52,7 @@ def test_config0_lockstep_full():
     cfg = configs.get(0)
     s = make_setup(cfg)
     prompts = corpus.make_prompts(cfg, 1)
-    check(lockstep(s, prompts, cfg.max_new, cfg.k, **F32_TOL))
+    check(lockstep(s, prompts, cfg.max_new, cfg.k, **F32_TOL), "config0 B=1 full")
 
 
 @pytest.mark.gpu
@@ -37,7 +60,7 @@ def test_config0_batch_with_gain_jitter_and_ragged_prompts():
     cfg = configs.get(0)
     s = make_setup(cfg, gain_jitter=0.2)
     prompts = corpus.make_prompts(cfg, 5, prompt_len=37)          # 37: prefill ends in a ragged chunk
-    check(lockstep(s, prompts, 24, 7, **F32_TOL))
+    check(lockstep(s, prompts, 24, 7, **F32_TOL), "config0 B=5 k=7 gain jitter ragged prompts")
 
 
 @pytest.mark.gpu
@@ -47,7 +70,7 @@ def test_config0_teacher_forced_accept_lengths():
     prompts = corpus.make_prompts(cfg, 3)
     for a in (0, 2, cfg.k):
         rep = lockstep(s, prompts, 20, cfg.k, oracle_kwargs=[dict(forced_accept=a)] * 3, forced_mode="accept", **F32_TOL)
-        check(rep)
+        check(rep, f"config0 forced accept {a}")
 
 
 @pytest.mark.gpu
@@ -75,11 +98,7 @@ def test_config0_generate_matches_oracle_and_plain_greedy(side_stream):
     assert sum(st.accepted_hist) > 0 and st.decode_ms > 0
     for i in range(B):
         spec = G.greedy_speculative(s.oracle, s.ngrams, prompts[i], cfg.max_new, cfg.k)
-        gaps = [g for stp in spec.steps for g in stp.gap]
-        want = np.array(spec.tokens)
-        if not np.array_equal(out[i], want):
-            first = int(np.argmax(out[i] != want))
-            assert min(gaps) < F32_TOL["gap_tol"], f"sequence {i} diverges at {first} without a near-tie"
+        assert_diverges_only_at_a_near_tie(out[i], spec, F32_TOL["gap_tol"], f"sequence {i}")
     # the committed tokens on the device equal the returned output
     tok = tokens.cpu().numpy()
     assert np.array_equal(tok[:, P:P + cfg.max_new], out)
@@ -136,14 +155,14 @@ def setup1():
 def test_config1_lockstep_batch1_full(setup1):
     cfg = configs.get(1)
     prompts = corpus.make_prompts(cfg, 1)
-    check(lockstep(setup1, prompts, cfg.max_new, cfg.k, **BF16_TOL))
+    check(lockstep(setup1, prompts, cfg.max_new, cfg.k, **BF16_TOL), "config1 B=1 full depth, 128 tokens")
 
 
 @pytest.mark.gpu
 def test_config1_lockstep_batch16_short(setup1):
     cfg = configs.get(1)
     prompts = corpus.make_prompts(cfg, 16)
-    check(lockstep(setup1, prompts, 12, cfg.k, **BF16_TOL))
+    check(lockstep(setup1, prompts, 12, cfg.k, **BF16_TOL), "config1 B=16 full depth, 12 tokens")
 
 
 @pytest.mark.gpu
@@ -153,7 +172,7 @@ def test_config1_teacher_forced_continuation(setup1):
     cont = corpus.make_continuations(cfg, prompts, 40 + cfg.k + 1)
     rep = lockstep(setup1, prompts, 40, cfg.k, oracle_kwargs=[dict(continuation=cont[i]) for i in range(2)],
                    forced_mode="continuation", **BF16_TOL)
-    check(rep)
+    check(rep, "config1 B=2 teacher-forced continuation")
 
 
 @pytest.mark.gpu
@@ -161,7 +180,7 @@ def test_config2_lockstep_short():
     cfg = configs.get(2)
     s = make_setup(cfg, n_docs=20000)
     prompts = corpus.make_prompts(cfg, 2)
-    check(lockstep(s, prompts, 18, 8, **BF16_TOL))
+    check(lockstep(s, prompts, 18, 8, **BF16_TOL), "config2 B=2 k=8 full depth, 18 tokens")
 
 
 @pytest.mark.gpu
@@ -186,7 +205,7 @@ def test_config3_expanded_vocabulary_lockstep():
     P = min(len(r) for r in re)
     prompts = np.stack([r[:P] for r in re]).astype(np.int32)
     assert prompts.max() >= base                      # merged tokens do occur in the prompts
-    check(lockstep(s, prompts, 12, cfg.k, **BF16_TOL))
+    check(lockstep(s, prompts, 12, cfg.k, **BF16_TOL), "config3 merged vocabulary, 2 layers, B=2")
 
 
 @pytest.mark.gpu
@@ -197,7 +216,7 @@ def test_config4_shape_long_context_lockstep():
     cfg = configs.shrunk(configs.get(4), n_layers=2, vocab=32768, n_docs=20000)
     s = make_setup(cfg)
     prompts = corpus.make_prompts(cfg, 2)
-    check(lockstep(s, prompts, 14, cfg.k, **BF16_TOL))
+    check(lockstep(s, prompts, 14, cfg.k, **BF16_TOL), "config4 geometry, 2 layers, B=2")
 
 
 @pytest.mark.gpu
@@ -245,7 +264,7 @@ def test_config2_batch32_k3_and_k8_one_step():
     s = make_setup(cfg)
     prompts = corpus.make_prompts(cfg, 32, prompt_len=80)
     for k in (3, 8):
-        check(lockstep(s, prompts, k + 1, k, **BF16_TOL))
+        check(lockstep(s, prompts, k + 1, k, **BF16_TOL), f"config2 geometry, 2 layers, B=32 k={k}")
 
 
 @pytest.mark.gpu
@@ -290,3 +309,140 @@ def test_a_wait_that_nothing_ends_times_out_and_leaves_the_context_usable():
     assert float(b.tasc_gemm_bf16(x, x).sum()) == 8 * 8 * 64
     with pytest.raises(b.TascError):
         b.tasc_selftest_bounded_wait(ws, 0)
+
+
+# ------------------------------------------------------------------------------------------ widest batch, full depth
+@pytest.mark.gpu
+def test_config4_geometry_batch64_k6_rows_0_1_63():
+    """Configuration 4's geometry at its benchmark batch: 64 sequences x (k + 1 = 7) rows = 448 GEMM rows (four token
+    tiles of 112, 224 accumulator columns per tile), prompts of 1,024 tokens, two layers, 32k vocabulary.  The oracle
+    runs sequences 0, 1 and 63; the other 61 decode along on the device."""
+    cfg = configs.shrunk(configs.get(4), n_layers=2, vocab=32768, n_docs=20000)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 64)
+    check(lockstep(s, prompts, 2 * (cfg.k + 1), cfg.k, oracle_rows=[0, 1, 63], **BF16_TOL),
+          "config4 geometry, 2 layers, B=64 k=6 (M=448), rows 0/1/63")
+
+
+@pytest.mark.gpu
+def test_config4_full_depth_batch1():
+    """The 1.5B shape at its full depth (28 layers, vocabulary 151,936, prompt of 1,024 tokens), one sequence,
+    four or more steps; the corpus tables come from the first 20,000 documents."""
+    cfg = configs.shrunk(configs.get(4), n_docs=20000)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 1)
+    check(lockstep(s, prompts, 4 * (cfg.k + 1), cfg.k, **BF16_TOL), "config4 full depth (28 layers), B=1, 28 tokens")
+
+
+@pytest.mark.gpu
+def test_config3_full_depth_batch1():
+    """The 0.5B shape with the merged vocabulary (V = 160,128) at its full depth of 24 layers, one sequence."""
+    from dataclasses import replace
+    from workload import vocab_expand as VE, weights as W
+    cfg3 = configs.shrunk(configs.get(3), n_docs=5000)
+    base = cfg3.model.vocab
+    toks, offs = corpus.make_corpus(cfg3)
+    merges = VE.select_merges(toks, offs, cfg3.n_merged_tokens, n_max=4, vocab=base)
+    toks2, offs2 = VE.retokenize(toks, offs, merges, vocab=base)
+    host_w = VE.expand_weights(W.make_weights(cfg3.model, cfg3.seed_weights), merges)
+    cfg = replace(cfg3, model=replace(cfg3.model, vocab=base + len(merges)))
+    s = make_setup(cfg, host_w=host_w, corpus_tokens=(toks2, offs2))
+    raw = corpus.make_prompts(cfg3, 1)
+    prompts = VE.retokenize(raw[0], np.array([0, raw.shape[1]]), merges, vocab=base)[0][None, :].astype(np.int32)
+    check(lockstep(s, prompts, 4 * (cfg.k + 1), cfg.k, **BF16_TOL), "config3 full depth (24 layers, V=160,128), B=1, 24 tokens")
+
+
+def one_step_from_prompts(b, s, prompts, drafts_h, k):
+    """Prefill + one verify step with the given drafts; returns (logits, targets, n_accepted, next) as numpy."""
+    B, P = prompts.shape
+    stride = P + 2 * (k + 1)
+    tokens = torch.zeros((B, stride), dtype=torch.int32, device="cuda")
+    tokens[:, :P] = torch.from_numpy(prompts).cuda()
+    length = torch.full((B,), P, dtype=torch.int32, device="cuda")
+    pool, bt, kv = s.model.new_kv(B, stride + b.MAX_ROWS)
+    ws = s.model.new_workspace(B, k)
+    seqs = b.make_seqs(tokens, length)
+    b.tasc_prefill(s.model, kv, seqs, B, P, ws)
+    n_acc, nxt, tgt, logits = b.tasc_verify_step(s.model, kv, seqs, torch.from_numpy(drafts_h).cuda(), ws,
+                                                 want_targets=True, want_logits=True)
+    b.tasc_poll_status(ws)
+    return logits.cpu().numpy(), tgt.cpu().numpy(), n_acc.cpu().numpy(), nxt.cpu().numpy()
+
+
+# A sequence's result must not depend on what else is in the batch.  It cannot be bit-identical: the number of
+# k-splits of a projection and of key-range splits of the attention is planned from the row count, so float32 sums
+# are associated differently at B = 1 and B = 16 / 64, and a K or V element that lands on the other side of a bf16
+# rounding boundary moves by 2^-9 of its value.  The bound is a quarter of the tolerance against the oracle.
+BATCH_INVARIANCE_ATOL = 5e-3
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("which,B,rows", [(1, 16, (0, 7, 15)), (4, 64, (0, 63))])
+def test_a_sequence_does_not_depend_on_its_batch(which, B, rows):
+    b = need_gpu()
+    if which == 1:
+        cfg = configs.shrunk(configs.get(1), n_docs=2000)                              # full depth: 30 layers
+    else:
+        cfg = configs.shrunk(configs.get(4), n_layers=2, vocab=32768, n_docs=2000)
+    s = make_setup(cfg, build_drafter=False, oracle_ngrams=False)
+    k = cfg.k
+    prompts = corpus.make_prompts(cfg, B)
+    drafts_h = np.random.default_rng(11).integers(0, cfg.model.vocab, (B, k)).astype(np.int32)
+    lg, tgt, n_acc, nxt = one_step_from_prompts(b, s, prompts, drafts_h, k)
+    worst = 0.0
+    for i in rows:
+        lg1, tgt1, n_acc1, nxt1 = one_step_from_prompts(b, s, prompts[i:i + 1], drafts_h[i:i + 1], k)
+        diff = float(np.abs(lg[i] - lg1[0]).max())
+        worst = max(worst, diff)
+        assert diff <= BATCH_INVARIANCE_ATOL, (i, diff)
+        top2 = np.sort(lg1[0], axis=-1)[:, -2:]
+        gap = top2[:, 1] - top2[:, 0]
+        for r in range(k + 1):
+            assert tgt[i, r] == tgt1[0, r] or gap[r] <= 2 * diff, (i, r, gap[r], diff)
+        if (tgt[i] == tgt1[0]).all():
+            assert n_acc[i] == n_acc1[0] and nxt[i] == nxt1[0]
+    print(f"batch invariance config {which} B={B}: max |logit difference| {worst:.3e}")
+
+
+@pytest.mark.gpu
+def test_whole_verify_step_is_bitwise_repeatable(setup1):
+    """The same step from the same state twice (split-K and the attention merge are reduced in a fixed order, the
+    LM-head maximum is order-free): logits, targets and the committed result must be bit-identical."""
+    b = need_gpu()
+    cfg = configs.get(1)
+    B, k = 16, cfg.k
+    prompts = corpus.make_prompts(cfg, B)
+    drafts_h = np.random.default_rng(3).integers(0, cfg.model.vocab, (B, k)).astype(np.int32)
+    first = one_step_from_prompts(b, setup1, prompts, drafts_h, k)
+    for _ in range(2):
+        again = one_step_from_prompts(b, setup1, prompts, drafts_h, k)
+        for x, y in zip(first, again):
+            assert np.array_equal(x, y)
+
+
+@pytest.mark.gpu
+def test_config1_generate_against_the_oracle(setup1):
+    """tasc_generate (bf16 model, graph-replayed steps) free-running against the oracle's speculative decoding:
+    a sequence may leave the oracle's tokens only at a token whose own oracle row was a near-tie."""
+    b = need_gpu()
+    cfg = configs.get(1)
+    B, max_new, k = 2, 48, cfg.k
+    prompts = corpus.make_prompts(cfg, B)
+    P = prompts.shape[1]
+    stride = P + max_new + k + 2
+    tokens = torch.zeros((B, stride), dtype=torch.int32, device="cuda")
+    tokens[:, :P] = torch.from_numpy(prompts).cuda()
+    length = torch.full((B,), P, dtype=torch.int32, device="cuda")
+    pool, bt, kv = setup1.model.new_kv(B, stride + b.MAX_ROWS)
+    ws = setup1.model.new_workspace(B, k)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        out, st = b.tasc_generate(setup1.model, setup1.drafter, kv, b.make_seqs(tokens, length), B, max_new, k, ws)
+    torch.cuda.current_stream().wait_stream(stream)
+    out = out.cpu().numpy()
+    diverged = []
+    for i in range(B):
+        spec = G.greedy_speculative(setup1.oracle, setup1.ngrams, prompts[i], max_new, k)
+        diverged.append(assert_diverges_only_at_a_near_tie(out[i], spec, BF16_TOL["gap_tol"], f"sequence {i}"))
+    print(f"config 1 free-running generation: first divergence per sequence {diverged} (None = identical {max_new} tokens)")
