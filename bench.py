@@ -42,7 +42,12 @@ UNIT = "tokens/s"
 # DRAM traffic of the fused GEMM kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum summed
 # over the step's launches of that kernel, per launch), keyed by (configuration, batch, k).  A figure is valid for
 # the kernel source whose digest is stored with it; after any change of gemm_fused.cu `traffic` reads null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # configuration 4, B = 1, k = 6: per layer 6.48 + 4.92 + 55.21 + 28.20 MB (QKV, O, gate/up, down) and 469.8 MB for the LM
+    # head, captured on the same kernels with the model cut to 2 layers (--layers 2) and summed for 28 layers, over the
+    # step's 113 launches (algorithmic: 27.55 MB per launch)
+    (4, 1, 6): {"bytes_per_launch": (28 * (6478592 + 4917248 + 55210496 + 28198912) + 469819904) / 113, "kernel_sha256_16": "401ea28c23a8b0b2"},
+}
 
 
 def kernel_digest():
@@ -258,27 +263,47 @@ class Task:
         host_w = W.make_weights(shape, cfg.seed_weights)
         ctoks, coffs = corpus.make_corpus(cfg, n_docs=corpus_docs)
         prompts_all = corpus.make_prompts(cfg, n_prompts)
+        dev_w = b.weights_to_device(host_w, shape.dtype, dev)
+        self.tokenizer = None
         if cfg.n_merged_tokens:
-            # configuration 3: merged n-gram tokens on top of the vocabulary (rows = constituent means), corpus and
-            # prompts re-tokenised by greedy longest match; selection from the first 20,000 documents
+            # configuration 3: the vocabulary is enriched on the device (Algorithm 1 of the paper on the first 20,000
+            # documents, n-grams of up to 4 tokens), the new embedding / LM-head rows are the means of their constituents,
+            # and corpus and prompts are re-encoded by longest match with the added tokens first
             from dataclasses import replace
-            from workload import vocab_expand as VE
             base = shape.vocab
             sel = min(len(coffs) - 1, 20000)
-            merges = VE.select_merges(ctoks[:coffs[sel]], coffs[:sel + 1], cfg.n_merged_tokens, n_max=4, vocab=base)
-            host_w = VE.expand_weights(host_w, merges)
-            ctoks, coffs = VE.retokenize(ctoks, coffs, merges, vocab=base)
-            re = [VE.retokenize(pr, np.array([0, pr.size]), merges, vocab=base)[0] for pr in prompts_all]
-            plen = min(len(r) for r in re)
-            prompts_all = np.stack([r[:plen] for r in re]).astype(np.int32)
-            shape = replace(shape, vocab=base + len(merges))
+            t0 = time.perf_counter()
+            merges, _, _ = b.tasc_tok_enrich(torch.from_numpy(ctoks[:coffs[sel]]).to(dev), torch.from_numpy(coffs[:sel + 1]).to(dev),
+                                             base, cfg.n_merged_tokens, 4)
+            torch.cuda.synchronize()
+            t_enrich = time.perf_counter() - t0
+            rows = b.tasc_tok_init_rows(dev_w["embed"], merges)
+            tied = dev_w["lm_head"] is dev_w["embed"]
+            lm_rows = rows if tied else b.tasc_tok_init_rows(dev_w["lm_head"], merges)
+            dev_w["embed"] = torch.cat([dev_w["embed"], rows]).contiguous()
+            dev_w["lm_head"] = dev_w["embed"] if tied else torch.cat([dev_w["lm_head"], lm_rows]).contiguous()
+            n_before = int(ctoks.size)
+            enc_t, enc_o = b.tasc_tok_encode(torch.from_numpy(ctoks).to(dev), torch.from_numpy(coffs).to(dev), base, merges)
+            ctoks, coffs = enc_t.cpu().numpy(), enc_o.cpu().numpy()
+            P0 = prompts_all.shape[1]
+            p_t, p_o = b.tasc_tok_encode(torch.from_numpy(prompts_all.reshape(-1).astype(np.int32)).to(dev),
+                                         torch.arange(0, prompts_all.size + 1, P0, dtype=torch.int64, device=dev), base, merges)
+            p_t, p_o = p_t.cpu().numpy(), p_o.cpu().numpy()
+            plen = int(np.diff(p_o).min())
+            prompts_all = np.stack([p_t[p_o[i]:p_o[i] + plen] for i in range(prompts_all.shape[0])]).astype(np.int32)
+            shape = replace(shape, vocab=base + int(merges.shape[0]))
+            self.tokenizer = {"added_tokens": int(merges.shape[0]), "enrich_s": t_enrich, "selection_documents": sel,
+                              "corpus_tokens_before": n_before, "corpus_tokens_after": int(ctoks.size),
+                              "compression": n_before / max(int(ctoks.size), 1)}
+            host_w = None
         self.shape, self.prompts_all = shape, prompts_all
-        self.model = b.Model(shape, b.weights_to_device(host_w, shape.dtype, dev), max_positions=cfg.prompt_len + cfg.max_new + 4096,
-                             page_size=cfg.page_size)
+        self.model = b.Model(shape, dev_w, max_positions=cfg.prompt_len + cfg.max_new + 4096, page_size=cfg.page_size)
         self.host_w = host_w if keep_host_weights else None
         del host_w
         # the corpus tables (once per task): built once untimed (allocator, module load), then timed with the corpus resident
         d_ctoks, d_coffs = torch.from_numpy(ctoks).to(dev), torch.from_numpy(coffs).to(dev)
+        # the output variability of the task corpus (Section 3 of the paper), reported next to the speed figures
+        self.corpus_stats = b.tasc_corpus_stats(d_ctoks, d_coffs, shape.vocab)
         drafter = b.tasc_drafter_build(d_ctoks, d_coffs, cfg.n_max, cfg.p_min, shape.vocab)
         del drafter
         torch.cuda.synchronize()
@@ -578,7 +603,9 @@ def main():
     cpu = None
     if want_cpu:
         n_seq, n_st = (1, 6) if shape.matmul_params() > 1e9 else (2, 12)
-        v, cores, desc, _ = oracle_sample(cfg, n_seq, n_st, k, task.prompts_all[:n_seq], host_w=task.host_w)
+        # (the enriched-vocabulary configuration is timed on the base vocabulary: the oracle's step cost is the same)
+        cpu_prompts = corpus.make_prompts(cfg, n_seq) if cfg.n_merged_tokens else task.prompts_all[:n_seq]
+        v, cores, desc, _ = oracle_sample(cfg, n_seq, n_st, k, cpu_prompts, host_w=task.host_w)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
     task.host_w = None
 
@@ -626,7 +653,8 @@ def main():
                        "parallelism": "replicas only (independent batches per GPU, no collective)" if world > 1 else "single GPU"},
             "mean_committed_per_step": committed_all / (args.steps * B * world),
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-            "generate": gen, "drafter_build": task.build_report, "workloads": workloads,
+            "generate": gen, "drafter_build": task.build_report, "corpus_statistics": task.corpus_stats,
+            "tokenizer_enrichment": task.tokenizer, "workloads": workloads,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -188,7 +188,7 @@ def lockstep(s: Setup, prompts: np.ndarray, max_new: int, k: int, *, logit_atol:
                 rep.max_logit_err = max(rep.max_logit_err, float(err.max()))
                 rep.max_err_over_or_bound = max(rep.max_err_over_or_bound,
                                                 float((err / np.maximum(logit_atol, logit_rtol * np.abs(ref))).max()))
-                bad = err > logit_atol + logit_rtol * np.abs(ref)
+                bad = err > np.maximum(logit_atol, logit_rtol * np.abs(ref))      # within the absolute OR the relative bound
                 if bad.any():
                     rep.hard_mismatches.append(("logits", step, i, float(err.max())))
             if row_ok or forced_mode is not None:

@@ -8,7 +8,8 @@ from oracle import decode as G
 from tests.gpu_harness import lockstep, make_setup, need_gpu, record_parity
 from workload import configs, corpus
 
-# logits tolerance: float32 model 1e-4 absolute; bf16 models max-abs 2e-2 / relative 1e-2.
+# logits tolerance: float32 model 1e-4 absolute; bf16 models max-abs 2e-2 or relative 1e-2 (an element passes if it is
+# within either bound: |err| <= max(2e-2, 1e-2 |ref|)).
 # token rule: a device argmax may differ from the oracle's only where the oracle's top-2 gap is below gap_tol.
 F32_TOL = dict(logit_atol=1e-4, logit_rtol=0.0, gap_tol=2e-4)
 BF16_TOL = dict(logit_atol=2e-2, logit_rtol=1e-2, gap_tol=1e-2)
@@ -251,7 +252,7 @@ def test_bf16_prefill_of_ragged_lengths_in_wide_passes():
         s.oracle.prefill(host[i, :L - 1], cache)
         st = G.verify_step(s.oracle, cache, int(host[i, L - 1]), list(map(int, drafts_h[i])), keep_logits=True)
         err = np.abs(lg[i] - st.logits)
-        assert (err <= BF16_TOL["logit_atol"] + BF16_TOL["logit_rtol"] * np.abs(st.logits)).all(), (i, float(err.max()))
+        assert (err <= np.maximum(BF16_TOL["logit_atol"], BF16_TOL["logit_rtol"] * np.abs(st.logits))).all(), (i, float(err.max()))
         for r in range(k + 1):
             assert int(tgt[i, r]) == st.y[r] or st.gap[r] < BF16_TOL["gap_tol"], (i, r)
 
