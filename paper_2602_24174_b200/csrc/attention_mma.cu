@@ -95,12 +95,18 @@ __device__ __forceinline__ void pack_hilo(float x, float y, uint32_t& hi, uint32
 // bandwidth; a shallower ring lets two CTAs share an SM when many (sequence, KV head) pairs are in flight.
 template <int HD, int NS> struct Ring { static constexpr int MAX_STAGES = HD >= 128 ? (NS > 4 ? 4 : 5) : 8; };
 
-// Warp groups of an eight-warp CTA whose query tile has n_slabs slabs and whose key range has n_tiles tiles: as many
-// groups as the warps allow, provided that each keeps two ring stages (one computing, one in flight) -- or that the
-// whole range fits the ring at once, in which case nothing is streamed behind the computation anyway.
+// Warp groups of an eight-warp CTA whose query tile has n_slabs slabs and whose key range has n_tiles tiles.  With a
+// single slab four groups work on four key tiles at once whatever the ring depth allows behind them: a ring of one
+// filling per group (the next tiles requested only once these are used) still beats two groups with a tile in flight
+// (ceil(T/4) x 3 us against ceil(T/2) x 2 us for T tiles of 128-wide heads).  With more slabs the SM's mma.sync pipes are
+// busy anyway, and each group keeps two ring stages (one computing, one in flight) unless the whole range fits at once.
 __host__ __device__ inline int warp_groups(int n_slabs, int stages, int n_tiles) {
     int ng = 8 / n_slabs;
     ng = ng >= 4 ? 4 : (ng >= 2 ? 2 : 1);
+    if (n_slabs == 1) {
+        while (ng > 1 && stages / ng < 1) ng >>= 1;
+        return ng;
+    }
     while (ng > 1 && stages / ng < 2 && !(stages / ng >= 1 && n_tiles <= (stages / ng) * ng)) ng >>= 1;
     return ng;
 }
@@ -173,11 +179,12 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         return;
     }
     const int total = pos0 + rows;               // keys visible to the last row
-    int chunk = (total + a.splits - 1) / a.splits;
-    chunk = (chunk + TKEYS - 1) / TKEYS * TKEYS;
-    const int k_begin = sp * chunk;
-    const int k_end = min(total, k_begin + chunk);
-    const int n_tiles = k_begin < k_end ? (k_end - k_begin + TKEYS - 1) / TKEYS : 0;
+    // the range's 64-key tiles are dealt out evenly: every split gets floor or ceil of tiles / splits of them
+    const int tiles_all = (total + TKEYS - 1) / TKEYS;
+    const int t_base = tiles_all / a.splits, t_rem = tiles_all % a.splits;
+    const int n_tiles = t_base + (sp < t_rem ? 1 : 0);
+    const int k_begin = (sp * t_base + min(sp, t_rem)) * TKEYS;
+    const int k_end = min(total, k_begin + n_tiles * TKEYS);
     const int n_slabs = (G + 15) / 16;
     // A warp owns one 16-row slab of one key tile.  With fewer slabs than warps the warps form ng = 2 or 4 groups
     // of n_slabs warps; group `grp` handles tiles grp, grp + ng, ...; the groups' results are merged in shared memory.
