@@ -89,6 +89,17 @@ tasc_status tasc_drafter_build(const int32_t* corpus_tokens, const int64_t* doc_
 tasc_status tasc_drafter_export(const tasc_drafter* d, tasc_ngram_entry* out, int64_t cap, int64_t* n_entries,
                                 int32_t* fallback_token);
 
+/*
+ * The inverse of tasc_drafter_export: a drafter handle from the surviving elements of the pruned models (any order of
+ * the entries; a duplicate (n, ctx, next) is an error the call does not detect) and the last-resort token.  Used to
+ * save a built drafter and load it again without the corpus.
+ *   entries  host, n_entries of them;  n_max 1..TASC_MAX_ORDER;  every id in [0, vocab), every count >= 1
+ *   out      host; receives a handle owning device tables (tasc_drafter_destroy)
+ * Synchronises the stream.  Errors: EINVAL, ENOMEM, ECUDA.
+ */
+tasc_status tasc_drafter_import(const tasc_ngram_entry* entries, int64_t n_entries, int32_t n_max, int32_t vocab,
+                                int32_t fallback_token, tasc_stream stream, tasc_drafter** out);
+
 tasc_status tasc_drafter_destroy(tasc_drafter* d);
 
 /*

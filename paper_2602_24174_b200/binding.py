@@ -83,6 +83,8 @@ lib.tasc_last_error.restype = C.c_char_p
 lib.tasc_drafter_build.argtypes = [_P, _P, C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(_P)]
 lib.tasc_drafter_export.argtypes = [_P, C.POINTER(NgramEntry), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 lib.tasc_drafter_destroy.argtypes = [_P]
+lib.tasc_drafter_import.argtypes = [C.POINTER(NgramEntry), C.c_int64, C.c_int32, C.c_int32, C.c_int32, _P, C.POINTER(_P)]
+lib.tasc_drafter_import.restype = C.c_int32
 lib.tasc_drafter_from_bigram.argtypes = [_P, C.c_int32, _P, C.POINTER(_P)]
 lib.tasc_drafter_from_bigram.restype = C.c_int32
 lib.tasc_bigram_table.argtypes = [_P, C.POINTER(Kv), C.c_int32, _P, _P, C.c_size_t, _P]
@@ -179,6 +181,18 @@ def tasc_drafter_build(corpus_tokens: torch.Tensor, doc_offsets: torch.Tensor, n
     h = _P()
     _check(lib.tasc_drafter_build(_ptr(corpus_tokens), _ptr(doc_offsets), doc_offsets.numel() - 1, n_max, p_min, vocab,
                                   _stream(), C.byref(h)), "tasc_drafter_build")
+    return Drafter(h, n_max)
+
+
+def tasc_drafter_import(entries: np.ndarray, fallback: int, n_max: int, vocab: int) -> Drafter:
+    """Drafter handle from the array Drafter.export() returns (int64[E, MAX_ORDER + 3] rows n, ctx, next, count)."""
+    entries = np.asarray(entries, dtype=np.int64).reshape(-1, MAX_ORDER + 3)
+    buf = (NgramEntry * max(len(entries), 1))()
+    raw = np.frombuffer(buf, dtype=np.int32).reshape(-1, MAX_ORDER + 3)
+    raw[:len(entries), :MAX_ORDER + 2] = entries[:, :MAX_ORDER + 2]
+    raw[:len(entries), MAX_ORDER + 2] = entries[:, MAX_ORDER + 2].astype(np.uint32).view(np.int32)
+    h = _P()
+    _check(lib.tasc_drafter_import(buf, len(entries), n_max, vocab, fallback, _stream(), C.byref(h)), "tasc_drafter_import")
     return Drafter(h, n_max)
 
 

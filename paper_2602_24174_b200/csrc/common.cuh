@@ -197,7 +197,7 @@ __device__ __forceinline__ void split_bf16(float v, __nv_bfloat16& hi, __nv_bflo
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-// ---------------------------------------------------------------- TMA (tiled bulk tensor load, no multicast)
+// ---------------------------------------------------------------- TMA (tiled bulk tensor load into this CTA only)
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }

@@ -765,6 +765,88 @@ extern "C" tasc_status tasc_drafter_export(const tasc_drafter* d, tasc_ngram_ent
     return w == total ? TASC_OK : TASC_ECAPACITY;
 }
 
+extern "C" tasc_status tasc_drafter_import(const tasc_ngram_entry* entries, int64_t n_entries, int32_t n_max, int32_t vocab,
+                                           int32_t fallback_token, tasc_stream stream_, tasc_drafter** out) {
+    if (!out) return TASC_EINVAL;
+    *out = nullptr;
+    if (n_entries < 0 || (n_entries > 0 && !entries) || n_max < 1 || n_max > TASC_MAX_ORDER || vocab < 1 ||
+        vocab > (1 << TASC_VOCAB_BITS) || fallback_token < 0 || fallback_token >= vocab)
+        return TASC_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // the packed (context, next) keys and counts of every order, in the form the build's compaction kernels read
+    std::vector<std::vector<uint64_t>> keys((size_t)n_max + 1);
+    std::vector<std::vector<uint32_t>> counts((size_t)n_max + 1);
+    for (int64_t i = 0; i < n_entries; ++i) {
+        const tasc_ngram_entry& e = entries[i];
+        if (e.n < 1 || e.n > n_max || e.next < 0 || e.next >= vocab || e.count < 1) return TASC_EINVAL;
+        Key k = key_make(e.n);
+        for (int j = 0; j < e.n; ++j) {
+            if (e.ctx[j] < 0 || e.ctx[j] >= vocab) return TASC_EINVAL;
+            key_put(k, j, (uint32_t)e.ctx[j]);
+        }
+        key_put(k, e.n, (uint32_t)e.next);
+        keys[e.n].push_back(k.lo);
+        keys[e.n].push_back(k.hi);
+        counts[e.n].push_back(e.count);
+    }
+    tasc_drafter* d = new (std::nothrow) tasc_drafter();
+    if (!d) return TASC_ENOMEM;
+    for (int n = 0; n <= TASC_MAX_ORDER; ++n) d->dt.t[n] = OrderTable{nullptr, nullptr, nullptr, 0, 0};
+    d->dt.n_max = n_max; d->dt.fallback = fallback_token; d->p_min = 1; d->vocab = vocab;
+    cudaGetDevice(&d->device);
+    tasc_status rc = TASC_OK;
+    int* status = nullptr;
+    unsigned long long* cursor = nullptr;
+    if (cudaMalloc(reinterpret_cast<void**>(&status), sizeof(int)) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&cursor), sizeof(unsigned long long)) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ENOMEM; }
+    if (rc == TASC_OK) cudaMemsetAsync(status, 0, sizeof(int), stream);
+    for (int n = 1; n <= n_max && rc == TASC_OK; ++n) {
+        const uint64_t cnt = counts[n].size();
+        if (cnt == 0) continue;
+        uint64_t* skeys = nullptr;
+        uint32_t *scounts = nullptr, *fill = nullptr;
+        OrderTable& t = d->dt.t[n];
+        const uint64_t ccap = pow2_at_least(2 * cnt);
+        t.mask = ccap - 1;
+        t.n_succ = (long long)cnt;
+        if (cudaMalloc(reinterpret_cast<void**>(&skeys), cnt * 16) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&scounts), cnt * 4) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&fill), ccap * 4) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&t.keys), ccap * 16) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&t.vals), ccap * sizeof(CtxVal)) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&t.succ), cnt * sizeof(Succ)) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ENOMEM; }
+        if (rc == TASC_OK) {
+            cudaMemcpyAsync(skeys, keys[n].data(), cnt * 16, cudaMemcpyHostToDevice, stream);
+            cudaMemcpyAsync(scounts, counts[n].data(), cnt * 4, cudaMemcpyHostToDevice, stream);
+            cudaMemsetAsync(t.keys, 0, ccap * 16, stream);
+            cudaMemsetAsync(t.vals, 0, ccap * sizeof(CtxVal), stream);
+            cudaMemsetAsync(fill, 0, ccap * 4, stream);
+            cudaMemsetAsync(cursor, 0, sizeof(unsigned long long), stream);
+            ctx_insert_kernel<<<blocks_for(cnt, 256), 256, 0, stream>>>(skeys, scounts, cnt, 1u, n, t, status);
+            assign_offsets_kernel<<<blocks_for(ccap, 256), 256, 0, stream>>>(t, cursor);
+            succ_fill_kernel<<<blocks_for(cnt, 256), 256, 0, stream>>>(skeys, scounts, cnt, 1u, n, t, fill, status);
+            if (cudaStreamSynchronize(stream) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ECUDA; }
+        }
+        if (skeys) cudaFree(skeys);
+        if (scounts) cudaFree(scounts);
+        if (fill) cudaFree(fill);
+    }
+    if (rc == TASC_OK) {
+        int st = 0;
+        if (cudaMemcpy(&st, status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { (void)cudaGetLastError(); rc = TASC_ECUDA; }
+        else if (st != 0) rc = st;
+    }
+    if (status) cudaFree(status);
+    if (cursor) cudaFree(cursor);
+    if (rc != TASC_OK) {
+        free_tables(d->dt);
+        delete d;
+        return rc;
+    }
+    *out = d;
+    return TASC_OK;
+}
+
 extern "C" tasc_status tasc_drafter_destroy(tasc_drafter* d) {
     if (!d) return TASC_EINVAL;
     free_tables(d->dt);

@@ -162,3 +162,26 @@ def test_config4_corpus_slice_tables_at_order_5():
     assert_tables_equal(dr, ng)
     ctxs = draft_contexts(cfg, tokens, offsets, 24, 600, seed=4)
     assert_drafts_equal(b, dr, ng, ctxs, cfg.k, [(3, 4), (1, 1)], stride=640)
+
+
+@pytest.mark.gpu
+def test_export_then_import_gives_the_same_drafter():
+    """A drafter rebuilt from its own canonical export (without the corpus) exports the same entries and drafts the same."""
+    cfg = configs.get(0)
+    tokens, offsets = corpus.make_corpus(cfg, n_docs=1200)
+    b, dr, ng = build_both(tokens, offsets, cfg.n_max, cfg.p_min, cfg.model.vocab)
+    ent, fb = dr.export()
+    r = np.random.default_rng(0)
+    dr2 = b.tasc_drafter_import(ent[r.permutation(len(ent))], fb, cfg.n_max, cfg.model.vocab)      # any order of the entries
+    ent2, fb2 = dr2.export()
+    assert fb2 == fb and np.array_equal(ent2, ent)
+    assert_tables_equal(dr2, ng)
+    ctxs = draft_contexts(cfg, tokens, offsets, 48, 100, seed=7)
+    assert_drafts_equal(b, dr2, ng, ctxs, cfg.k, [(3, 4), (1, 1), (0, 1)], stride=128)
+    empty = b.tasc_drafter_import(np.zeros((0, D.MAX_ORDER + 3), np.int64), 5, 3, 16)
+    ent3, fb3 = empty.export()
+    assert fb3 == 5 and len(ent3) == 0
+    bad = ent.copy()
+    bad[0, D.MAX_ORDER + 1] = cfg.model.vocab                                                      # next token outside the vocabulary
+    with pytest.raises(b.TascError):
+        b.tasc_drafter_import(bad, fb, cfg.n_max, cfg.model.vocab)
