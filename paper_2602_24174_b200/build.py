@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libtasc.so")
-SOURCES = ["api.cu", "drafter.cu", "gemm_tcgen05.cu", "gemm_fused.cu", "attention_mma.cu", "gemm_simt.cu", "gemm_static.cu", "tasc_tok.cu", "layers.cu", "attention.cu", "profile.cu"]
+SOURCES = ["api.cu", "drafter.cu", "gemm_tcgen05.cu", "gemm_fused.cu", "gemm_wide.cu", "attention_mma.cu", "gemm_simt.cu", "gemm_static.cu", "tasc_tok.cu", "layers.cu", "attention.cu", "profile.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -33,6 +33,7 @@ struct tasc_model {
     CUtensorMap tm_lm;
     int qkv_rows, q_dim, kv_dim;
     int few_tiles;                                  // token tiles for 49..128 rows (see gemm_token_tile), from the layer's weight bytes
+    double layer_mb;                                // projection weights of one layer, MB
     mutable std::mutex plan_mu;
     mutable std::vector<StepPlans> plans;           // most recently used last; a handful of (B, k, workspace) combinations
 };
@@ -123,7 +124,7 @@ Workspace layout_workspace(const tasc_model* m, int B, void* base_) {
     const size_t att_bytes = d.dtype == TASC_F32 ? attention_scratch_bytes(B, TASC_MAX_ROWS, d.n_q_heads, d.head_dim, splits_max) : ALIGN;
     w.att_scratch = L.take<float>(base, att_bytes / sizeof(float));
     w.ssq_slots = (d.d_model + 127) / 128;
-    w.ssq = L.take<float>(base, M * w.ssq_slots);
+    w.ssq = L.take<float>(base, M * w.ssq_slots * 4);      // passes of more than 128 rows keep four slots per 128 features
     w.bytes = L.off;
     return w;
 }
@@ -147,6 +148,15 @@ KvView layer_kv(const tasc_model* m, const tasc_kv* kv, int layer) {
 }
 
 // Where the rows of a forward come from: a verify step (chunk < 0: last committed token + drafts) or prefill chunk `chunk`.
+// Which passes and products take the many-row kernel (gemm_wide.cu); see plan_fused.  Measured on the 135M, 0.5B and
+// 1.5B shapes at 192 .. 1,024 rows: a product gains from it once its weight matrix has about 7 MB (gate/up, down and
+// the LM head of the larger shapes; the narrow QKV and O matrices stay with the few-row kernel and its 128-row weight
+// tiles), and a pass of 129 .. 255 rows only on layers of 60 MB and more (its two token tiles fill three quarters of
+// the MMA's rows or less, and the few-row kernel then prefers three narrower tiles).
+constexpr double WIDE_MATRIX_MB = 7.0;
+constexpr double WIDE_LAYER_MB = 60.0;
+constexpr int WIDE_ROWS = 256;
+
 struct RowSource {
     const tasc_seqs* seqs;
     const int32_t* drafts;
@@ -216,16 +226,20 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
             // attention works on blocks of at most 16 rows per sequence (one block in a verify step, several in a prefill pass)
             const int att_rows = R <= 16 ? R : 16;
             sp.att = plan_attention_mma(B * (R / att_rows), d.n_kv_heads, d.head_dim, d.n_q_heads / d.n_kv_heads, att_rows, max_ctx);
-            sp.TB = gemm_token_tile(M, true, m->few_tiles);
+            // passes of more than 128 rows: the products with large weight matrices take the many-row kernel
+            const double big_mb = 2.0 * 2.0 * (double)d.d_ff * d.d_model / 1e6;      // the largest matrix of a layer (gate/up)
+            const bool wide_pass = M > 128 && big_mb >= WIDE_MATRIX_MB && (M >= WIDE_ROWS || m->layer_mb >= WIDE_LAYER_MB);
+            const double wide_min_mb = wide_pass ? WIDE_MATRIX_MB : -1.0;
+            sp.TB = gemm_token_tile(M, true, m->few_tiles, wide_min_mb >= 0.0);
             sp.rows = (uint64_t)((M + sp.TB - 1) / sp.TB) * 2 * sp.TB;
             if ((st = encode_tmap_bf16(&sp.tm_h, w.h, sp.rows, d.d_model, 2 * sp.TB)) != TASC_OK) return st;
             if ((st = encode_tmap_bf16(&sp.tm_o, w.o, sp.rows, m->q_dim, 2 * sp.TB)) != TASC_OK) return st;
             if ((st = encode_tmap_bf16(&sp.tm_act, w.act, sp.rows, d.d_ff, 2 * sp.TB)) != TASC_OK) return st;
-            sp.p_qkv = plan_fused(M, m->qkv_rows, d.d_model, EPI_QKV, m->few_tiles);
-            sp.p_o = plan_fused(M, d.d_model, m->q_dim, EPI_RESID, m->few_tiles);
-            sp.p_gu = plan_fused(M, d.d_ff, d.d_model, EPI_SWIGLU, m->few_tiles);
-            sp.p_down = plan_fused(M, d.d_model, d.d_ff, EPI_RESID, m->few_tiles);
-            sp.p_lm = plan_fused(M, d.vocab, d.d_model, EPI_LM, m->few_tiles);
+            sp.p_qkv = plan_fused(M, m->qkv_rows, d.d_model, EPI_QKV, m->few_tiles, d.head_dim, wide_min_mb);
+            sp.p_o = plan_fused(M, d.d_model, m->q_dim, EPI_RESID, m->few_tiles, 0, wide_min_mb);
+            sp.p_gu = plan_fused(M, d.d_ff, d.d_model, EPI_SWIGLU, m->few_tiles, 0, wide_min_mb);
+            sp.p_down = plan_fused(M, d.d_model, d.d_ff, EPI_RESID, m->few_tiles, 0, wide_min_mb);
+            sp.p_lm = plan_fused(M, d.vocab, d.d_model, EPI_LM, m->few_tiles, 0, wide_min_mb);
             // the LM head's CTAs take several layout tiles at once
             if ((st = encode_tmap_bf16(&sp.tm_h_lm, w.h, sp.rows, d.d_model, sp.p_lm.BN)) != TASC_OK) return st;
             if (m->plans.size() >= 16) m->plans.erase(m->plans.begin());
@@ -242,13 +256,16 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
 
     FusedArgs base = {};
     base.M = M;
-    base.ssq_slots = w.ssq_slots;
+    const int ssq_sub = M > 128 ? 4 : 1;
+    const int ssq_slots = w.ssq_slots * ssq_sub;
+    base.ssq_slots = ssq_slots;
+    base.ssq_sub = ssq_sub;
     base.inv_d = 1.0f / (float)d.d_model;
     base.eps = d.rms_eps;
     base.status = w.status;
 
     launch_rows_embed(w.rp, src.seqs->tokens, src.seqs->stride, src.seqs->len, src.seqs->stop_len, src.drafts, B, R, src.chunk,
-                      d.vocab, w.status, static_cast<const __nv_bfloat16*>(m->embed), m->attn_norm[0], w.x, h, w.ssq, w.ssq_slots,
+                      d.vocab, w.status, static_cast<const __nv_bfloat16*>(m->embed), m->attn_norm[0], w.x, h, w.ssq, ssq_slots,
                       lm_head ? w.argmax : nullptr, d.d_model, TB, s);
     for (int l = 0; l < d.n_layers; ++l) {
         const KvView kvl = layer_kv(m, kv, l);
@@ -267,7 +284,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
         if (st != TASC_OK) return st;
 
         a = base;
-        a.N = d.d_model; a.K = m->q_dim; a.x = w.x; a.gain = m->mlp_norm[l]; a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = w.ssq_slots;
+        a.N = d.d_model; a.K = m->q_dim; a.x = w.x; a.gain = m->mlp_norm[l]; a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = ssq_slots;
         a.early = 1;                   // x was last written three launches back
         if ((st = launch_gemm_fused(EPI_RESID, &m->tm_o[l], &tm_o, a, p_o, s)) != TASC_OK) return st;
 
@@ -277,7 +294,7 @@ tasc_status forward_bf16(const tasc_model* m, const tasc_kv* kv, const Workspace
 
         a = base;
         a.N = d.d_model; a.K = d.d_ff; a.x = w.x; a.gain = l + 1 < d.n_layers ? m->attn_norm[l + 1] : m->final_norm;
-        a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = w.ssq_slots;
+        a.a_out = h; a.ssq_out = w.ssq; a.ssq_out_slots = ssq_slots;
         a.early = 1;                   // x was last written two launches back
         if ((st = launch_gemm_fused(EPI_RESID, &m->tm_down[l], &tm_act, a, p_down, s)) != TASC_OK) return st;
     }
@@ -364,6 +381,7 @@ extern "C" tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc
         // exchange and epilogue time per layer: below 24 MB three tiles, below 60 MB two, above that one
         const double layer_mb = 2.0 * ((double)m->qkv_rows * d.d_model + (double)d.d_model * m->q_dim + 3.0 * d.d_ff * d.d_model) / 1e6;
         m->few_tiles = layer_mb < 24.0 ? 3 : (layer_mb < 60.0 ? 2 : 1);
+        m->layer_mb = layer_mb;
     }
     m->rope = nullptr;
     for (int l = 0; l < d.n_layers; ++l) {

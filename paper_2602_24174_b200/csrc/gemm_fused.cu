@@ -228,7 +228,11 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 store_hilo4(a.a_out + row * a.N + f, a.a_out + (row + TBL) * a.N + f, v);
             }
             ss = warp_sum(ss);
-            if (lane == 0) a.ssq_out[(size_t)m * a.ssq_out_slots + out_tile] = ss;
+            if (lane == 0) {
+                float* slot = a.ssq_out + (size_t)m * a.ssq_out_slots + (size_t)out_tile * a.ssq_sub;
+                slot[0] = ss;
+                for (int j = 1; j < a.ssq_sub; ++j) slot[j] = 0.f;
+            }
         } else if (EPI == EPI_SWIGLU) {
             const float sc = s_inv[t];
             // lanes 0-15 hold four gate features each, lanes 16-31 the matching up features: after the exchange both
@@ -620,9 +624,14 @@ tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const Fus
 
 }  // namespace
 
-FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles) {
-    FusedPlan p;
-    p.TBL = gemm_token_tile(M, true, few_tiles);
+FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles, int hd, double wide_min_mb) {
+    FusedPlan p = {};
+    const bool many_rows = wide_min_mb >= 0.0 && M > 128;
+    const double mb = 2.0 * (double)(epi == EPI_SWIGLU ? 2 * N : N) * (double)K / 1e6;
+    // (from 512 rows on, matrices of a little more than half that size gain as well)
+    if (many_rows && (mb >= wide_min_mb || (M >= 512 && mb >= 0.55 * wide_min_mb)) && plan_wide(M, N, K, epi, hd, p)) return p;
+    p = {};
+    p.TBL = gemm_token_tile(M, true, few_tiles, many_rows);
     // The LM head streams the largest matrix once and has no split-K exchange: one CTA takes as many layout tiles
     // as an MMA holds (256 columns), so that a weight tile is fetched by one CTA, not by one per token tile.
     const int span = epi == EPI_LM ? std::max(1, std::min((M + p.TBL - 1) / p.TBL, 128 / p.TBL)) : 1;
@@ -691,6 +700,7 @@ FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles) {
 tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
                               cudaStream_t stream) {
     if (a.M <= 0 || a.N <= 0 || a.K <= 0) return TASC_EINVAL;
+    if (p.wide) return launch_gemm_wide(epi, tmW, tmX, a, p, stream);
     a.num_kb = p.num_kb; a.BN = p.BN; a.TB = p.TB; a.TBL = p.TBL; a.stages = p.stages; a.pair = 1; a.data_bytes = p.data_bytes;
     switch (epi) {
         case EPI_PLAIN:  return launch_epi<EPI_PLAIN>(tmW, tmX, a, p, K_GEMM, stream);

@@ -216,7 +216,7 @@ tasc_status encode_tmap_kv(CUtensorMap* map, const void* ptr, uint64_t rows, int
     return r == CUDA_SUCCESS ? TASC_OK : TASC_ECUDA;
 }
 
-int gemm_token_tile(int M, bool pair, int few_tiles) {
+int gemm_token_tile(int M, bool pair, int few_tiles, bool many_rows) {
     const int cap = pair ? 128 : 256;                 // tokens per tile (UMMA N <= 256)
     int m_tiles = (M + cap - 1) / cap;
     // An MMA over a 128-row weight tile takes the same time for any number of token columns, while the split-K
@@ -224,9 +224,11 @@ int gemm_token_tile(int M, bool pair, int few_tiles) {
     // streams the weight tile again.  Which wins depends on the size of the weights: for narrow models (a few MB per
     // layer) three or more token tiles per weight tile run faster than one or two wide ones above 48 rows (measured at
     // 96, 192 and 448 rows); for a 94 MB layer one tile of 112 rows beats three of 48 by 20 % of the step, and in
-    // between two tiles are slightly ahead.  The caller passes the count for 49..128 rows (few_tiles); above 128 rows
-    // it stays at three or more.
-    if (pair && M > 48) m_tiles = std::max(m_tiles, M <= 128 ? std::max(1, std::min(few_tiles, 3)) : 3);
+    // between two tiles are slightly ahead.  The caller passes the count for 49..128 rows (few_tiles).  Above 128 rows
+    // it stays at three or more -- unless the pass runs its large products through the many-row kernel (gemm_wide.cu),
+    // where the token rows are the MMA's M (many_rows): then as few tiles of at most 128 rows as hold them.
+    if (pair && M > 48 && M <= 128) m_tiles = std::max(m_tiles, std::max(1, std::min(few_tiles, 3)));
+    if (pair && M > 128 && !many_rows) m_tiles = std::max(m_tiles, 3);
     const int per = (M + m_tiles - 1) / m_tiles;
     return std::max(16, (per + 15) / 16 * 16);
 }

@@ -33,7 +33,7 @@ struct GemmPlan {
 };
 GemmPlan plan_gemm(int M, int N, int K, size_t max_partial_bytes, bool pair);
 // TB for M token rows.  few_tiles (1..3): how many token tiles 49..128 paired rows are cut into at least (see gemm_token_tile).
-int gemm_token_tile(int M, bool pair, int few_tiles = 3);
+int gemm_token_tile(int M, bool pair, int few_tiles = 3, bool many_rows = false);
 inline size_t gemm_partial_bytes(const GemmPlan& p, int M, int N) { return (size_t)p.splits * M * N * sizeof(float); }
 
 // rows x cols bf16 row-major matrix, box = {64 cols, box_rows}, 128-byte swizzle.
@@ -58,6 +58,7 @@ enum Epi {
 struct FusedArgs {
     int M, N, K;                       // token rows, output features (EPI_SWIGLU: d_ff), reduction length
     int num_kb, BN, TB, TBL, stages, pair, data_bytes; // filled in by launch_gemm_fused from the plan
+    int BNW, n_ft, n_tt;               // many-row kernel (gemm_wide.cu): features per MMA, feature tiles, token tiles
     int early;                         // the epilogue's global operands were complete before the preceding grid began
     const float* ssq_in;               // [M][ssq_slots] partial sums of squares of the input rows (null: no scaling)
     int ssq_slots;
@@ -74,7 +75,8 @@ struct FusedArgs {
     float* x;                          // EPI_RESID
     const float* gain;
     float* ssq_out;
-    int ssq_out_slots;
+    int ssq_out_slots;                 // slots per row; ssq_sub of them per 128 features (the many-row kernel writes one per 32 features)
+    int ssq_sub;
     __nv_bfloat16* a_out;              // EPI_RESID / EPI_SWIGLU: activation buffer of the next GEMM, [tiles][2 TB][N]
     unsigned long long* argmax;        // EPI_LM
     float* logits;
@@ -85,8 +87,17 @@ struct FusedPlan {
     int TB, BN, m_tiles, out_tiles, num_kb;   // TB: tokens per CTA (a multiple of TBL); BN = 2 TB; m_tiles: CTAs along the tokens
     int S;             // cluster size = k-splits
     int stages, data_bytes, smem_bytes;
+    int wide;          // 1: the many-row kernel of gemm_wide.cu (M > 128) with BNW weight rows per MMA and `grid` persistent CTAs
+    int BNW, grid;
 };
-FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles = 3);
+// hd: head_dim, for EPI_QKV.  wide_min_mb: < 0 for a pass whose products all take the few-row kernel; otherwise the
+// pass lays its activations out for the many-row kernel (gemm_token_tile with many_rows) and a product takes that
+// kernel if its weight matrix has at least this many MB.
+FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles = 3, int hd = 0, double wide_min_mb = -1.0);
+// The many-row variant (gemm_wide.cu): fills `p` and returns true where it applies (M > 128, N a multiple of 32).
+bool plan_wide(int M, int N, int K, int epi, int hd, FusedPlan& p);
+tasc_status launch_gemm_wide(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
+                             cudaStream_t stream);
 // tmW: weight map with box rows 128 (64 for EPI_SWIGLU); tmX: (hi, lo) activation map with box rows BN = 2 TB.
 tasc_status launch_gemm_fused(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
                               cudaStream_t stream);

@@ -326,6 +326,23 @@ def test_config4_geometry_batch64_k6_rows_0_1_63():
 
 
 @pytest.mark.gpu
+def test_many_row_kernel_on_every_product_with_64_wide_heads():
+    """A one-layer shape whose five weight matrices are all large enough for the many-row GEMM kernel (d_model 2,048,
+    32 query / 8 KV heads of 64, d_ff 2,048, vocabulary 8,192: 8 to 34 MB each) at 40 sequences x 7 rows = 280 rows
+    (three token tiles of 96) after a prefill in passes of 640 rows: its QKV epilogue with two RoPE halves of 32 per
+    head, the split-K clusters of the narrow products, the residual and SiLU epilogues and the row arg-max.  The oracle
+    runs sequences 0 and 39."""
+    from dataclasses import replace
+    base = configs.shrunk(configs.get(2), n_docs=3000)
+    shape = replace(base.model, n_layers=1, d_model=2048, n_q_heads=32, n_kv_heads=8, head_dim=64, d_ff=2048, vocab=8192)
+    cfg = replace(base, model=shape)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, 40, prompt_len=80)
+    check(lockstep(s, prompts, 2 * (cfg.k + 1), 6, oracle_rows=[0, 39], **BF16_TOL),
+          "many-row kernel, 1 layer, d_model 2048, heads of 64, B=40 k=6 (M=280)")
+
+
+@pytest.mark.gpu
 def test_config4_full_depth_batch1():
     """The 1.5B shape at its full depth (28 layers, vocabulary 151,936, prompt of 1,024 tokens), one sequence,
     four or more steps; the corpus tables come from the first 20,000 documents."""
