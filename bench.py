@@ -336,7 +336,14 @@ class Window:
         self.kvs = task.model.new_kv(B, self.stride + b.MAX_ROWS, dev)
         self.seqs = b.make_seqs(self.tokens, self.length)
         self.drafts = torch.empty((B, k), dtype=torch.int32, device=dev)
-        b.tasc_prefill(task.model, self.kvs[2], self.seqs, B, P, self.ws)
+        b.tasc_prefill(task.model, self.kvs[2], self.seqs, B, P, self.ws)       # first call: plans, attributes
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        b.tasc_prefill(task.model, self.kvs[2], self.seqs, B, P, self.ws)       # the same prompts again, timed
+        e1.record()
+        torch.cuda.synchronize()
+        self.prefill_ms = e0.elapsed_time(e1)
         for _ in range(warmup):
             self.one_step()
         b.tasc_poll_status(self.ws)
@@ -620,7 +627,11 @@ def main():
             return {"workload": f"config {t.cfg.index} ({t.cfg.name}) B={Bw} k={kw} prompt {pw.shape[1]}", "steps": steps,
                     "ms_per_step": ms_w / steps, "tokens_per_s_window": com_w / (ms_w * 1e-3),
                     "mean_committed_per_step": com_w / (steps * Bw), "bound": r["bound"], "frac": r["frac"],
-                    "achieved": r["achieved"], "unit": r["unit"], "bytes_per_step": r["bytes_per_step"], "roofline_us": r["roofline_us"]}
+                    "achieved": r["achieved"], "unit": r["unit"], "bytes_per_step": r["bytes_per_step"], "roofline_us": r["roofline_us"],
+                    "gemm_rows_per_step": Bw * (kw + 1), "prefill_ms": w.prefill_ms,
+                    # the prefill runs the layers, not the LM head, over all but the last prompt token
+                    "prefill_tflops": 2.0 * (t.shape.matmul_params() - t.shape.vocab * t.shape.d_model) * Bw * (pw.shape[1] - 1)
+                                      / (w.prefill_ms * 1e-3) / 1e12}
 
         def corpus_prompts(t, Bw):
             if t.prompts_all.shape[0] >= Bw:
@@ -630,13 +641,13 @@ def main():
             if cfg.index == 4 and Bw != B:
                 workloads.append(sub_record(task, Bw, k, 48))
         del win
-        for ci, batches in ((2, (1, 8)), (1, (1, 16))):
+        for ci, runs in ((2, ((1, 5), (8, 5), (32, 5), (32, 8))), (1, ((1, 5), (16, 5)))):
             if ci == cfg.index:
                 continue
             c = configs.get(ci)
-            t = Task(b, c, dev, max(batches), corpus_docs=min(c.corpus.n_docs, 50000))
-            for Bw in batches:
-                workloads.append(sub_record(t, Bw, c.k, 64))
+            t = Task(b, c, dev, max(Bw for Bw, _ in runs), corpus_docs=min(c.corpus.n_docs, 50000))
+            for Bw, kw in runs:
+                workloads.append(sub_record(t, Bw, kw, 64))
             del t
             torch.cuda.empty_cache()
 

@@ -277,7 +277,8 @@ tasc_status tasc_model_create(const tasc_model_desc* desc, const tasc_weights* w
 tasc_status tasc_model_destroy(tasc_model* m);
 
 /* Bytes of workspace that step calls need for up to B_max sequences and k_max drafts.  bf16 models reserve
- * room for at least 1,024 rows in flight, which prefill passes of few sequences use (tens of MB at most). */
+ * room for at least 2,048 rows in flight, which prefill passes use (up to 256 rows per sequence; 140 MB for the
+ * 1.5B shape, tens of MB for the small ones). */
 size_t tasc_workspace_bytes(const tasc_model* m, int32_t B_max, int32_t k_max);
 
 /*

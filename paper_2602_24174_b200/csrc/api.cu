@@ -73,7 +73,7 @@ struct Workspace {
 
 // Rows a pass may carry: TASC_MAX_ROWS per sequence for a verify step, and for bf16 models at least PREFILL_ROWS
 // in all, so that a prefill of few sequences still runs passes of hundreds of rows (weights are read once per pass).
-constexpr int PREFILL_ROWS = 1024;
+constexpr int PREFILL_ROWS = 2048;
 constexpr int PREFILL_ROWS_PER_SEQ = 256;
 size_t workspace_rows(const tasc_model* m, int B) {
     const size_t verify = (size_t)B * TASC_MAX_ROWS;
