@@ -326,6 +326,19 @@ def test_config4_geometry_batch64_k6_rows_0_1_63():
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("B", [19, 32])
+def test_config4_geometry_between_one_and_two_full_token_tiles(B):
+    """Configuration 4's geometry (two layers, 32k vocabulary) at 19 and 32 sequences x 7 rows: 133 rows = two token
+    tiles of 80 whose second holds 53 rows (a ragged tail in the many-row kernel's last tile), and 224 rows = two full
+    tiles of 112.  The oracle runs the first and the last sequence."""
+    cfg = configs.shrunk(configs.get(4), n_layers=2, vocab=32768, n_docs=20000)
+    s = make_setup(cfg)
+    prompts = corpus.make_prompts(cfg, B, prompt_len=200)
+    check(lockstep(s, prompts, cfg.k + 1, cfg.k, oracle_rows=[0, B - 1], **BF16_TOL),
+          f"config4 geometry, 2 layers, B={B} k=6 (M={B * 7}), rows 0/{B - 1}")
+
+
+@pytest.mark.gpu
 def test_many_row_kernel_on_every_product_with_64_wide_heads():
     """A one-layer shape whose five weight matrices are all large enough for the many-row GEMM kernel (d_model 2,048,
     32 query / 8 KV heads of 64, d_ff 2,048, vocabulary 8,192: 8 to 34 MB each) at 40 sequences x 7 rows = 280 rows
