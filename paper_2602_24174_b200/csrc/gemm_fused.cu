@@ -26,7 +26,9 @@
 // touches activations, and releases the next grid once its last weight load has been issued.
 //
 // Warp roles (192 threads): warps 0-3 epilogue (TMEM lane quarter w), warp 4 TMA producer, warp 5
-// TMEM allocation + MMA issue.  Every mbarrier wait is bounded; a wait that runs out records
+// TMEM allocation + MMA issue; all of them reduce and finish token columns afterwards.  Where a CTA
+// finishes a dozen columns or more, that part is bound by instruction latency (one warp per scheduler),
+// and the launch carries six more warps (384 threads) that do nothing else.  Every mbarrier wait is bounded; a wait that runs out records
 // TASC_ETIMEOUT, the CTA still takes part in the cluster barriers, frees its TMEM and returns.
 #include "kernels.h"
 
@@ -42,7 +44,9 @@ constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
-constexpr int THREADS = 192;
+constexpr int THREADS = 192;                  // six warps; launches with many token columns per CTA add six more that only finish columns
+constexpr int MAX_THREADS = 384;
+constexpr int FINISHERS_MIN_COLS = 12;
 constexpr int MAX_DYN_SMEM = 226 * 1024;      // 227 KB per CTA minus the kernel's static shared memory
 
 #ifdef TASC_TIMELINE
@@ -83,7 +87,7 @@ __device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, const float v[4])
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(MAX_THREADS, 1)
 gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const FusedArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -148,7 +152,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     // first NPF columns of every warp are fetched while the MMAs run, so their latency is off the tail.
     struct Pre { float4 x, cs01, cs23; int pos, page; };
     constexpr int NPF = 3;
-    constexpr int EW = 6;                       // all six warps reduce and finish columns (column tl belongs to warp tl % 6)
+    const int EW = (int)(blockDim.x >> 5);      // every warp (6 or 12) reduces and finishes columns: column tl belongs to warp tl % EW
     auto prefetch = [&](int tl) -> Pre {
         Pre q;
         q.x = q.cs01 = q.cs23 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -354,6 +358,11 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             TL(5);
         }
         __syncwarp();
+        griddep_wait();
+        if (!a.early) late_prefetch();
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ the additional column finishers: nothing to do before part 2
+        if (a.early) late_prefetch();
         griddep_wait();
         if (!a.early) late_prefetch();
     } else {
@@ -600,7 +609,7 @@ tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const Fus
     if (pst != TASC_OK) return pst;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.S, (unsigned)p.out_tiles, (unsigned)p.m_tiles);
-    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.blockDim = dim3((unsigned)(p.threads == MAX_THREADS ? MAX_THREADS : THREADS), 1, 1);
     cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute at[2];
@@ -694,6 +703,11 @@ FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles, int hd, double
         const int fit = max_active_clusters_any(epi, S, p.smem_bytes);
         if (fit <= 0 || tiles <= fit) break;
     }
+    // token columns a CTA reduces and finishes after the cluster exchange
+    const int cols_cta = (std::min(p.TB, M) + p.S - 1) / p.S;
+    // (only for grids of one wave: with two CTAs per SM the schedulers have warps enough, and twelve warps of 100 to 126
+    // registers would not leave room for the second CTA)
+    p.threads = (epi != EPI_LM && epi != EPI_PLAIN && cols_cta >= FINISHERS_MIN_COLS && tiles * p.S <= 148) ? MAX_THREADS : THREADS;
     return p;
 }
 

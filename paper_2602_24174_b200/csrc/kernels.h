@@ -89,6 +89,7 @@ struct FusedPlan {
     int stages, data_bytes, smem_bytes;
     int wide;          // 1: the many-row kernel of gemm_wide.cu (M > 128) with BNW weight rows per MMA and `grid` persistent CTAs
     int BNW, grid;
+    int threads;       // few-row kernel: 192, or 384 (six more warps that only finish columns) where a CTA finishes many token columns
 };
 // hd: head_dim, for EPI_QKV.  wide_min_mb: < 0 for a pass whose products all take the few-row kernel; otherwise the
 // pass lays its activations out for the many-row kernel (gemm_token_tile with many_rows) and a product takes that
