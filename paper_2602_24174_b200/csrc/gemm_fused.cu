@@ -86,8 +86,9 @@ __device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, const float v[4])
     *reinterpret_cast<uint2*>(p) = u;
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
+// EW: warps of the CTA (6, or 12 with the additional column finishers); all of them reduce and finish columns.
+template <int EPI, int EW>
+__global__ void __launch_bounds__(EW * 32, 1)
 gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const FusedArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -152,7 +153,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     // first NPF columns of every warp are fetched while the MMAs run, so their latency is off the tail.
     struct Pre { float4 x, cs01, cs23; int pos, page; };
     constexpr int NPF = 3;
-    const int EW = (int)(blockDim.x >> 5);      // every warp (6 or 12) reduces and finishes columns: column tl belongs to warp tl % EW
+    // every warp reduces and finishes columns: column tl belongs to warp tl % EW
     auto prefetch = [&](int tl) -> Pre {
         Pre q;
         q.x = q.cs01 = q.cs23 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -554,7 +555,8 @@ tasc_status prepare_epi() {
     TASC_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return TASC_EINVAL;
     if (!attr_done[dev]) {
-        TASC_CUDA_TRY(cudaFuncSetAttribute(gemm_fused_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM));
+        TASC_CUDA_TRY(cudaFuncSetAttribute(gemm_fused_kernel<EPI, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM));
+        TASC_CUDA_TRY(cudaFuncSetAttribute(gemm_fused_kernel<EPI, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN_SMEM));
         attr_done[dev] = true;
     }
     return TASC_OK;
@@ -576,7 +578,7 @@ int max_active_clusters(int S, int smem) {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_fused_kernel<EPI>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_fused_kernel<EPI, 6>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
     return n;
 }
 
@@ -627,7 +629,8 @@ tasc_status launch_epi(const CUtensorMap* tmW, const CUtensorMap* tmX, const Fus
     cfg.attrs = at;
     cfg.numAttrs = n;
     ProfScope ps(kind, stream);
-    TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_fused_kernel<EPI>, *tmW, *tmX, a));
+    if (p.threads == MAX_THREADS) TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_fused_kernel<EPI, 12>, *tmW, *tmX, a));
+    else TASC_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_fused_kernel<EPI, 6>, *tmW, *tmX, a));
     return TASC_OK;
 }
 
