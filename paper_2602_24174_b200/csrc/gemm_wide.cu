@@ -282,8 +282,12 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
         float sc = 1.0f;
         if (a.ssq_in && rowok) {
             float ss = 0.f;
-            const float4* sp = reinterpret_cast<const float4*>(a.ssq_in + (size_t)m * a.ssq_slots);   // a multiple of four slots
-            for (int q = 0; q < a.ssq_slots / 4; ++q) { const float4 t = sp[q]; ss += (t.x + t.y) + (t.z + t.w); }
+            if (a.ssq_slots % 4 == 0) {
+                const float4* sp = reinterpret_cast<const float4*>(a.ssq_in + (size_t)m * a.ssq_slots);
+                for (int q = 0; q < a.ssq_slots / 4; ++q) { const float4 t = sp[q]; ss += (t.x + t.y) + (t.z + t.w); }
+            } else {
+                for (int q = 0; q < a.ssq_slots; ++q) ss += a.ssq_in[(size_t)m * a.ssq_slots + q];
+            }
             sc = 1.0f / sqrtf(ss * a.inv_d + a.eps);
         }
 
@@ -643,11 +647,11 @@ int sm_count() {
 
 }  // namespace
 
-bool plan_wide(int M, int N, int K, int epi, int hd, FusedPlan& p) {
-    if (M <= 128 || N % 32 || K % 8) return false;
+bool plan_wide(int M, int N, int K, int epi, int hd, FusedPlan& p, int token_tile) {
+    if ((M <= 128 && token_tile <= 0) || N % 32 || K % 8) return false;
     if (epi != EPI_QKV && epi != EPI_RESID && epi != EPI_SWIGLU && epi != EPI_LM) return false;
     if (epi == EPI_QKV && hd != 64 && hd != 128) return false;
-    p.TBL = gemm_token_tile(M, true, 3, true);
+    p.TBL = token_tile > 0 ? token_tile : gemm_token_tile(M, true, 3, true);
     p.TB = p.TBL;
     p.BN = 2 * p.TBL;
     p.m_tiles = (M + p.TBL - 1) / p.TBL;

@@ -96,7 +96,8 @@ struct FusedPlan {
 // kernel if its weight matrix has at least this many MB.
 FusedPlan plan_fused(int M, int N, int K, int epi, int few_tiles = 3, int hd = 0, double wide_min_mb = -1.0);
 // The many-row variant (gemm_wide.cu): fills `p` and returns true where it applies (M > 128, N a multiple of 32).
-bool plan_wide(int M, int N, int K, int epi, int hd, FusedPlan& p);
+// token_tile > 0: the pass's token tile is given (its other products take the few-row kernel), any M.
+bool plan_wide(int M, int N, int K, int epi, int hd, FusedPlan& p, int token_tile = 0);
 tasc_status launch_gemm_wide(int epi, const CUtensorMap* tmW, const CUtensorMap* tmX, FusedArgs a, const FusedPlan& p,
                              cudaStream_t stream);
 // tmW: weight map with box rows 128 (64 for EPI_SWIGLU); tmX: (hi, lo) activation map with box rows BN = 2 TB.

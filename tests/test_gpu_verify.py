@@ -326,11 +326,12 @@ def test_config4_geometry_batch64_k6_rows_0_1_63():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("B", [19, 32])
+@pytest.mark.parametrize("B", [16, 19, 32])
 def test_config4_geometry_between_one_and_two_full_token_tiles(B):
-    """Configuration 4's geometry (two layers, 32k vocabulary) at 19 and 32 sequences x 7 rows: 133 rows = two token
-    tiles of 80 whose second holds 53 rows (a ragged tail in the many-row kernel's last tile), and 224 rows = two full
-    tiles of 112.  The oracle runs the first and the last sequence."""
+    """Configuration 4's geometry (two layers, 32k vocabulary) at 16, 19 and 32 sequences x 7 rows: 112 rows = one token
+    tile, where the layers take the few-row kernel (with its additional column finishers) and the LM head the many-row
+    kernel; 133 rows = two token tiles of 80 whose second holds 53 rows (a ragged tail in the many-row kernel's last
+    tile); 224 rows = two full tiles of 112.  The oracle runs the first and the last sequence."""
     cfg = configs.shrunk(configs.get(4), n_layers=2, vocab=32768, n_docs=20000)
     s = make_setup(cfg)
     prompts = corpus.make_prompts(cfg, B, prompt_len=200)
