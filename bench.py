@@ -46,7 +46,7 @@ NCU_TRAFFIC = {
     # configuration 4, B = 1, k = 6: per layer 6.48 + 4.92 + 55.21 + 28.20 MB (QKV, O, gate/up, down) and 469.8 MB for the LM
     # head, captured on the same kernels with the model cut to 2 layers (--layers 2) and summed for 28 layers, over the
     # step's 113 launches (algorithmic: 27.55 MB per launch)
-    (4, 1, 6): {"bytes_per_launch": (28 * (6478080 + 4911616 + 55202304 + 28193536) + 470263296) / 113, "kernel_sha256_16": "083e98412509ccb0"},
+    (4, 1, 6): {"bytes_per_launch": (28 * 94798336 + 470330624) / 113, "kernel_sha256_16": "73c53c5da55f6b57"},
 }
 
 
